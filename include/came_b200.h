@@ -1,0 +1,195 @@
+/*
+ * came_b200.h -- C ABI of the B200 (sm_100a) CAME optimizer step.
+ *
+ * The library performs one thing: the per-step parameter update of the CAME
+ * optimizer ("CAME: Confidence-guided Adaptive Memory Efficient Optimization",
+ * Algorithm 2) over a list of parameter tensors resident on one GPU.
+ *
+ * For a matrix parameter theta (n rows x m columns, row-major) with gradient g,
+ * one step computes, in the notation of Algorithm 2 (all matrix squares,
+ * divisions and roots element-wise, 1_n / 1_m all-ones vectors):
+ *
+ *   r_t = beta2 r_{t-1} + (1-beta2) (g^2 + eps1 1_n 1_m^T) 1_m        row sums
+ *   c_t = beta2 c_{t-1} + (1-beta2) 1_n^T (g^2 + eps1 1_n 1_m^T)      column sums
+ *   v_t = r_t c_t / 1_n^T r_t                                         (Eq. 2, rank one)
+ *   u_t = g / sqrt(v_t)
+ *   uhat_t = u_t / max(1, RMS(u_t)/d)                                 (Eq. 1)
+ *   m_t = beta1 m_{t-1} + (1-beta1) uhat_t
+ *   U_t = (uhat_t - m_t)^2
+ *   R_t = beta3 R_{t-1} + (1-beta3) (U_t + eps2 1_n 1_m^T) 1_m
+ *   C_t = beta3 C_{t-1} + (1-beta3) 1_n^T (U_t + eps2 1_n 1_m^T)
+ *   S_t = R_t C_t / 1_n^T R_t
+ *   theta_t = theta_{t-1} - eta (m_t / sqrt(S_t) + lambda theta_{t-1})
+ *
+ * r, c, R, C are EMAs of SUMS (not means), exactly as printed in Algorithm 2; a
+ * caller that keeps means converts with r_mean = r / m, c_mean = c / n.
+ * lambda (decoupled weight decay) is an extension: the paper has none, and
+ * lambda = 0 gives Algorithm 2 exactly.
+ *
+ * A vector parameter (ndim == 1) takes the unfactored path: v (stored in `r`)
+ * and S (stored in `R`) are full-length element-wise EMAs,
+ *   v_t = beta2 v + (1-beta2)(g^2 + eps1), u = g/sqrt(v_t), clip as above,
+ *   m_t as above, S_t = beta3 S + (1-beta3)((uhat - m_t)^2 + eps2),
+ *   theta_t = theta_{t-1} - eta (m_t / sqrt(S_t) + lambda theta_{t-1}),
+ * which is what Algorithm 2 yields for an n x 1 matrix.
+ *
+ * Initial state (inputs of Algorithm 2): m_0 = r_0 = c_0 = 0; R_0 = C_0 = 0 by
+ * the same convention.  came_create zero-fills the state unless told to keep it.
+ *
+ * Conventions for every entry point
+ *   - "device" pointers are CUDA device addresses on the context's GPU; "host"
+ *     pointers are ordinary process memory.  Each argument says which.
+ *   - The caller owns every tensor buffer it passes in; the library owns the
+ *     context and its internal device tables and reduction workspace.
+ *   - Every function returns a came_status; nothing is launched when
+ *     validation fails.  No exceptions, no abort.  came_last_error gives text.
+ *   - came_step enqueues work on the caller's stream and returns without
+ *     synchronising.  A context is not re-entrant: one thread at a time.
+ */
+#ifndef CAME_B200_H
+#define CAME_B200_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct came_ctx came_ctx;   /* opaque */
+
+typedef enum {
+    CAME_OK = 0,
+    CAME_ERR_NULL = 1,        /* a required pointer is NULL */
+    CAME_ERR_SHAPE = 2,       /* rows/cols/ndim/count out of range */
+    CAME_ERR_DTYPE = 3,       /* unknown gradient dtype */
+    CAME_ERR_ALIGN = 4,       /* a tensor pointer is not 16-byte aligned */
+    CAME_ERR_HPARAM = 5,      /* hyper-parameter out of range or not finite */
+    CAME_ERR_STEP_ORDER = 6,  /* step is not previous step + 1 */
+    CAME_ERR_DEVICE = 7,      /* bad device ordinal / no usable CUDA device */
+    CAME_ERR_OOM = 8,         /* host or device allocation failed */
+    CAME_ERR_CUDA = 9,        /* a CUDA runtime call failed; see came_last_error */
+    CAME_ERR_INTERNAL = 10,
+    CAME_ERR_UNSUPPORTED = 11 /* request outside what this entry point handles */
+} came_status;
+
+typedef enum { CAME_F32 = 0, CAME_BF16 = 1 } came_dtype;   /* gradient storage type */
+
+/* per-tensor flags */
+enum {
+    CAME_T_NO_WEIGHT_DECAY   = 1u << 0,  /* lambda treated as 0 for this tensor */
+    CAME_T_VEC_NO_CONFIDENCE = 1u << 1   /* vectors only: theta -= eta (m_t + lambda theta), i.e.
+                                            the last line of Algorithm 1; S is left untouched */
+};
+
+/* came_create flags */
+enum {
+    CAME_CREATE_KEEP_STATE = 1u << 0     /* resume: do not zero m, r, c, R, C */
+};
+
+/* One parameter tensor.  All pointers are DEVICE pointers, 16-byte aligned,
+ * to contiguous, non-overlapping buffers that stay valid until came_destroy. */
+typedef struct {
+    float*       param;   /* fp32 [rows*cols], row-major; updated in place              */
+    const void*  grad;    /* grad_dtype [rows*cols], same layout; read only             */
+    float*       m;       /* fp32 [rows*cols]  momentum of the clipped update           */
+    float*       r;       /* matrix: fp32 [rows] row factor of g^2 | vector: v [rows]    */
+    float*       c;       /* matrix: fp32 [cols] column factor     | vector: NULL        */
+    float*       R;       /* matrix: fp32 [rows] row factor of U   | vector: S [rows]    */
+    float*       C;       /* matrix: fp32 [cols] column factor     | vector: NULL        */
+    int64_t      rows;    /* >= 1 */
+    int64_t      cols;    /* >= 1; must be 1 when ndim == 1 */
+    int32_t      ndim;    /* 1 = vector, 2 = matrix; other ranks are not defined by the paper */
+    int32_t      grad_dtype;  /* came_dtype */
+    uint32_t     flags;   /* CAME_T_* */
+    uint32_t     reserved;    /* must be 0 */
+} came_tensor;
+
+/* Hyper-parameters of one step (doubles: 1-beta is formed in double, then each
+ * constant is rounded to fp32 once).  Symbols as in the inputs of Algorithm 2. */
+typedef struct {
+    double  lr;            /* eta    >= 0                                  */
+    double  beta1;         /* in [0,1)                                     */
+    double  beta2;         /* in [0,1)                                     */
+    double  beta3;         /* in [0,1)                                     */
+    double  eps1;          /* >= 0, regulariser of g^2                      */
+    double  eps2;          /* >= 0, regulariser of the instability U        */
+    double  clip_d;        /* d > 0, RMS clipping threshold (Eq. 1)         */
+    double  weight_decay;  /* lambda >= 0 (extension; 0 = the paper)        */
+    int64_t step;          /* t >= 1; must be previous + 1 after the first call.  Not used
+                              in the arithmetic (Algorithm 2 has no bias correction). */
+} came_hparams;
+
+/* came_query selectors */
+enum {
+    CAME_Q_NUMEL = 0,            /* total parameter elements                                    */
+    CAME_Q_STATE_BYTES = 1,      /* bytes of optimizer state m, r, c, R, C                       */
+    CAME_Q_STREAM_BYTES = 2,     /* algorithmic bytes per step when no tensor stays on chip      */
+    CAME_Q_COMPULSORY_BYTES = 3, /* floor: g, m, theta read once; m, theta written once          */
+    CAME_Q_WORKSPACE_BYTES = 4,  /* device bytes the context allocated                           */
+    CAME_Q_NUM_TILES = 5,        /* matrix tiles in the launch plan                              */
+    CAME_Q_LAUNCHES_PER_STEP = 6,/* kernels one came_step enqueues                               */
+    CAME_Q_LAST_STEP = 7,        /* last step accepted (0 before the first)                      */
+    CAME_Q_NUM_PHASES = 8,       /* entries came_get_phase_ms reports                            */
+    CAME_Q_MATRIX_NUMEL = 9      /* elements that live in matrices (the four-phase path)         */
+};
+
+/* Algorithm 2, set-up.  Validates `t[0..n)` (HOST array of descriptors holding
+ * DEVICE pointers), selects `device`, builds the launch plan, allocates the
+ * context's device tables and reduction workspace, and zero-fills the state
+ * buffers (m_0 = r_0 = c_0 = R_0 = C_0 = 0) unless CAME_CREATE_KEEP_STATE.
+ * Synchronises the device once.  On failure *out is NULL. */
+came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t device,
+                        uint32_t flags);
+
+/* Algorithm 2, one pass of the loop body over every tensor of the context.
+ * `hp`: HOST pointer.  `grads`: HOST array of n DEVICE gradient pointers that
+ * replace the ones given at create for this and later steps, or NULL to keep
+ * them.  `cuda_stream`: the caller's cudaStream_t (NULL = default stream).
+ * Asynchronous; allocates nothing. */
+came_status came_step(came_ctx* ctx, const came_hparams* hp, const void* const* grads,
+                      void* cuda_stream);
+
+/* Same step, fed from and drained to HOST memory: for every tensor i copies
+ * host_grads[i] (HOST, grad_dtype [rows*cols], ideally pinned) into the tensor's
+ * device gradient buffer, runs the step, then, where host_params_out is not NULL
+ * and host_params_out[i] is not NULL, copies the updated parameters back (HOST,
+ * fp32 [rows*cols]).  All on `cuda_stream`, asynchronous for pinned memory. */
+came_status came_step_host(came_ctx* ctx, const came_hparams* hp, const void* const* host_grads,
+                           void* const* host_params_out, void* cuda_stream);
+
+/* Frees the context's device and host memory.  Caller's tensors are untouched.
+ * The caller must have synchronised every stream it passed to came_step. */
+came_status came_destroy(came_ctx* ctx);
+
+/* Text of the last error on this context (or of the last failed came_create
+ * when ctx is NULL).  HOST string owned by the library. */
+const char* came_last_error(const came_ctx* ctx);
+
+/* Name of a status code.  HOST string, static. */
+const char* came_status_string(came_status s);
+
+/* Facts about the context; `what` is a CAME_Q_* selector, *out a HOST int64. */
+came_status came_query(const came_ctx* ctx, int32_t what, int64_t* out);
+
+/* Per-phase device timing.  When enabled, came_step records CUDA events on the
+ * caller's stream between its kernels (no synchronisation).  came_get_phase_ms
+ * synchronises on the last recorded event and writes up to `cap` durations in
+ * milliseconds (HOST floats) in launch order; names via came_phase_name. */
+came_status came_set_profiling(came_ctx* ctx, int32_t enabled);
+came_status came_get_phase_ms(came_ctx* ctx, float* out_ms, int32_t cap, int32_t* out_count);
+const char* came_phase_name(const came_ctx* ctx, int32_t phase);
+
+/* Launch-plan geometry of one tensor, computed on the host without touching
+ * the GPU (the same routine came_create uses).  Outputs (HOST): elements per
+ * thread per load (1, 4 or 8), threads across columns, rows per tile, number of
+ * row blocks and column blocks.  `aligned32` says whether param and m are
+ * 32-byte aligned; `tile_elems_target` <= 0 selects the default. */
+came_status came_plan_tensor(int64_t rows, int64_t cols, int32_t ndim, int32_t grad_dtype,
+                             int32_t aligned32, int64_t tile_elems_target, int32_t* out_vec,
+                             int32_t* out_threads_x, int32_t* out_tile_rows, int32_t* out_n_rb,
+                             int32_t* out_n_cb);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CAME_B200_H */

@@ -1,0 +1,642 @@
+// CAME optimizer step, device code for sm_100a.
+//
+// One step of Algorithm 2 has three grid-wide data dependencies per tensor
+// (r,c need all of g; the clip factor needs all of u; S needs all of U), so a
+// matrix is streamed in four phases, each one kernel over a multi-tensor tile
+// list:
+//   P1  g            -> row/column sums of g^2        -> r_t, c_t, sqrt(1^T r_t)
+//   P2  g, r, c      -> sum of u^2                    -> clip factor kappa (Eq. 1)
+//   P3  g, m, r, c   -> m_t, row/column sums of (uhat - m_{t-1})^2 -> R_t, C_t, sqrt(1^T R_t)
+//   P4  m, theta, R, C -> theta_t
+// v_t and S_t (Eq. 2, rank one) are never formed: u = g * rsqrt(r_i) * sqrt(sum r) * rsqrt(c_j),
+// which also keeps r_i * c_j out of fp32 (it underflows for zero-gradient rows).
+//
+// Reductions are deterministic: every tile writes its partial sums to a
+// workspace and the LAST tile to arrive (per row block, per column strip, per
+// tensor; counted with atomics) adds them in a fixed order.  No thread ever
+// waits on another block, so there is no spin anywhere in this file.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace came {
+
+constexpr int kThreads = 256;
+constexpr int kVecChunk = 4096;       // vector elements per block in the vector kernels
+
+enum Kind : int { kF32x4 = 0, kBF16x8 = 1, kF32x1 = 2, kBF16x1 = 3 };
+
+struct TensorDev {
+    float*       p;
+    const void*  g;
+    float*       m;
+    float*       r;      // vectors: v
+    float*       c;
+    float*       R;      // vectors: S
+    float*       C;
+    long long    rows, cols;
+    float*       ws_colpart;   // [n_rb][cols]   per-tile column partial sums
+    float*       ws_rowpart;   // [n_seg][rows]  per-warp-segment row partial sums
+    float*       ws_blocksum;  // [n_rb]         sum of the finished row factor over one row block
+    float*       ws_usq;       // [n_parts]      per-tile partial sums of u^2
+    unsigned*    cnt;          // [n_rb] row-block arrivals, [n_cb] strip arrivals, [1] finished, [1] usq
+    float*       scal;         // [0] sqrt(sum r)  [1] kappa  [2] sqrt(sum R)
+    int          kind;
+    int          vec;          // elements per thread per load
+    int          tx_log2;      // threads across columns = 1 << tx_log2 (32..256)
+    int          tr;           // rows per tile
+    int          n_rb, n_cb, n_seg;
+    int          n_parts;      // matrices: n_rb*n_cb; vectors: number of chunks
+    int          ndim;
+    unsigned     flags;
+};
+
+struct Tile { int tensor, rb, cb; };
+struct VChunk { int tensor, chunk; };
+
+struct StepConsts {
+    float beta1, omb1, b1sq;
+    float beta2, omb2;
+    float beta3, omb3;
+    float eps1, eps2;
+    float lr, wd;
+    float pad_;
+    double clip_d;
+};
+
+constexpr unsigned kFlagNoWd = 1u << 0;
+constexpr unsigned kFlagVecNoConf = 1u << 1;
+
+// ---------------------------------------------------------------------------
+// loads / stores
+// ---------------------------------------------------------------------------
+template <int KIND> struct Traits;
+template <> struct Traits<kF32x4>  { static constexpr int VEC = 4; };
+template <> struct Traits<kBF16x8> { static constexpr int VEC = 8; };
+template <> struct Traits<kF32x1>  { static constexpr int VEC = 1; };
+template <> struct Traits<kBF16x1> { static constexpr int VEC = 1; };
+
+__device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// gradient load: read-only for the whole step
+template <int KIND>
+__device__ __forceinline__ void load_g(const void* base, long long idx, float (&x)[Traits<KIND>::VEC])
+{
+    if constexpr (KIND == kF32x4) {
+        const float4 v = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(base) + idx));
+        x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
+    } else if constexpr (KIND == kBF16x8) {
+        const uint4 v = __ldg(reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(base) + idx));
+        x[0] = bf16lo(v.x); x[1] = bf16hi(v.x); x[2] = bf16lo(v.y); x[3] = bf16hi(v.y);
+        x[4] = bf16lo(v.z); x[5] = bf16hi(v.z); x[6] = bf16lo(v.w); x[7] = bf16hi(v.w);
+    } else if constexpr (KIND == kF32x1) {
+        x[0] = __ldg(static_cast<const float*>(base) + idx);
+    } else {
+        x[0] = __uint_as_float(static_cast<uint32_t>(__ldg(static_cast<const uint16_t*>(base) + idx)) << 16);
+    }
+}
+
+// fp32 state load/store: 1, 4 (128-bit) or 8 (256-bit, sm_100) floats per thread
+template <int VEC>
+__device__ __forceinline__ void load_f(const float* p, float (&x)[VEC])
+{
+    if constexpr (VEC == 8) {
+        asm volatile("ld.global.L1::no_allocate.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                     : "=f"(x[0]), "=f"(x[1]), "=f"(x[2]), "=f"(x[3]),
+                       "=f"(x[4]), "=f"(x[5]), "=f"(x[6]), "=f"(x[7]) : "l"(p));
+    } else if constexpr (VEC == 4) {
+        asm volatile("ld.global.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
+                     : "=f"(x[0]), "=f"(x[1]), "=f"(x[2]), "=f"(x[3]) : "l"(p));
+    } else {
+        x[0] = *p;
+    }
+}
+
+template <int VEC>
+__device__ __forceinline__ void store_f(float* p, const float (&x)[VEC])
+{
+    if constexpr (VEC == 8) {
+        asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                     :: "l"(p), "f"(x[0]), "f"(x[1]), "f"(x[2]), "f"(x[3]),
+                        "f"(x[4]), "f"(x[5]), "f"(x[6]), "f"(x[7]) : "memory");
+    } else if constexpr (VEC == 4) {
+        asm volatile("st.global.v4.f32 [%0], {%1,%2,%3,%4};"
+                     :: "l"(p), "f"(x[0]), "f"(x[1]), "f"(x[2]), "f"(x[3]) : "memory");
+    } else {
+        *p = x[0];
+    }
+}
+
+// ---------------------------------------------------------------------------
+// block-level helpers (deterministic: fixed shuffle tree, fixed warp order)
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+__device__ __forceinline__ double warp_sum(double v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+struct Shared {
+    float  colred[kThreads * 8];   // cross-row-group column reduction
+    double red[kThreads / 32];
+    int    flag[4];
+};
+
+// Sum over the block; result valid in every thread.  Two barriers.
+template <typename T>
+__device__ __forceinline__ T block_sum(T v, Shared& sm)
+{
+    v = warp_sum(v);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) sm.red[threadIdx.x >> 5] = static_cast<double>(v);
+    __syncthreads();
+    double s = 0.0;
+#pragma unroll
+    for (int w = 0; w < kThreads / 32; ++w) s += sm.red[w];
+    return static_cast<T>(s);
+}
+
+// ---------------------------------------------------------------------------
+// Last-arriver finalisation of one factored EMA (Algorithm 2: r_t, c_t from g^2
+// with beta2/eps1; R_t, C_t from U_t with beta3/eps2):
+//   row[i] = beta row[i] + (1-beta) (scale * sum_j X[i][j] + cols * eps)
+//   col[j] = beta col[j] + (1-beta) (scale * sum_i X[i][j] + rows * eps)
+// and, once every row block and strip of the tensor is finished,
+//   *sqrt_sum = sqrt(1_n^T row).
+// Called by every tile of the tensor after it has written its partials.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ void finalize_factors(const TensorDev& d, int rb, int cb, float beta,
+                                                 float omb, float eps, float scale,
+                                                 float* __restrict__ rowfac,
+                                                 float* __restrict__ colfac,
+                                                 float* __restrict__ sqrt_sum, Shared& sm)
+{
+    const int tid = threadIdx.x;
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const unsigned a = atomicAdd(&d.cnt[rb], 1u);
+        const unsigned b = atomicAdd(&d.cnt[d.n_rb + cb], 1u);
+        sm.flag[0] = (a == static_cast<unsigned>(d.n_cb - 1));
+        sm.flag[1] = (b == static_cast<unsigned>(d.n_rb - 1));
+    }
+    __syncthreads();
+    const bool last_r = sm.flag[0] != 0, last_c = sm.flag[1] != 0;
+    if (!last_r && !last_c) return;
+    __threadfence();
+
+    const long long rows = d.rows, cols = d.cols;
+    if (last_r) {
+        const long long row0 = static_cast<long long>(rb) * d.tr;
+        const long long row1 = min(rows, row0 + d.tr);
+        const float add = static_cast<float>(cols) * eps;
+        float bs = 0.f;
+        for (long long row = row0 + tid; row < row1; row += kThreads) {
+            float s = 0.f;
+            for (int sg = 0; sg < d.n_seg; ++sg) s += __ldcg(d.ws_rowpart + sg * rows + row);
+            const float nv = fmaf(beta, rowfac[row], omb * fmaf(scale, s, add));
+            rowfac[row] = nv;
+            bs += nv;
+        }
+        bs = block_sum(bs, sm);
+        if (tid == 0) { d.ws_blocksum[rb] = bs; d.cnt[rb] = 0u; }
+    }
+    if (last_c) {
+        const int sw = (1 << d.tx_log2) * d.vec;
+        const long long col0 = static_cast<long long>(cb) * sw;
+        const long long col1 = min(cols, col0 + sw);
+        const float add = static_cast<float>(rows) * eps;
+        for (long long col = col0 + tid; col < col1; col += kThreads) {
+            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+            const float* pc = d.ws_colpart + col;
+            int k = 0;
+            for (; k + 4 <= d.n_rb; k += 4) {      // fixed association, see the sum below
+                s0 += __ldcg(pc + (k + 0) * cols);
+                s1 += __ldcg(pc + (k + 1) * cols);
+                s2 += __ldcg(pc + (k + 2) * cols);
+                s3 += __ldcg(pc + (k + 3) * cols);
+            }
+            for (; k < d.n_rb; ++k) s0 += __ldcg(pc + k * cols);
+            const float s = (s0 + s1) + (s2 + s3);
+            colfac[col] = fmaf(beta, colfac[col], omb * fmaf(scale, s, add));
+        }
+        if (tid == 0) d.cnt[d.n_rb + cb] = 0u;
+    }
+    const unsigned done = (last_r ? 1u : 0u) + (last_c ? 1u : 0u);
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const unsigned a = atomicAdd(&d.cnt[d.n_rb + d.n_cb], done);
+        sm.flag[2] = (a + done == static_cast<unsigned>(d.n_rb + d.n_cb));
+    }
+    __syncthreads();
+    if (sm.flag[2]) {
+        __threadfence();
+        double s = 0.0;
+        for (int k = tid; k < d.n_rb; k += kThreads) s += static_cast<double>(__ldcg(d.ws_blocksum + k));
+        s = block_sum(s, sm);
+        if (tid == 0) { *sqrt_sum = static_cast<float>(sqrt(s)); d.cnt[d.n_rb + d.n_cb] = 0u; }
+    }
+}
+
+// Eq. 1: the last part to arrive adds all partial sums of u^2 in a fixed order
+// and stores kappa = 1 / max(1, RMS(u)/d), RMS over all rows*cols components.
+__device__ __forceinline__ void finalize_kappa(const TensorDev& d, int part, float partial,
+                                               double clip_d, Shared& sm)
+{
+    const int tid = threadIdx.x;
+    if (tid == 0) d.ws_usq[part] = partial;
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const unsigned a = atomicAdd(&d.cnt[d.n_rb + d.n_cb + 1], 1u);
+        sm.flag[3] = (a == static_cast<unsigned>(d.n_parts - 1));
+    }
+    __syncthreads();
+    if (!sm.flag[3]) return;
+    __threadfence();
+    double s = 0.0;
+    for (int k = tid; k < d.n_parts; k += kThreads) s += static_cast<double>(__ldcg(d.ws_usq + k));
+    s = block_sum(s, sm);
+    if (tid == 0) {
+        const double rms = sqrt(s / (static_cast<double>(d.rows) * static_cast<double>(d.cols)));
+        d.scal[1] = static_cast<float>(1.0 / fmax(1.0, rms / clip_d));
+        d.cnt[d.n_rb + d.n_cb + 1] = 0u;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// tile geometry shared by the four matrix phases
+// ---------------------------------------------------------------------------
+struct Geo {
+    int tx, ty, TY, seg;
+    long long col, row0, row1;
+    bool colok;
+};
+
+template <int VEC>
+__device__ __forceinline__ Geo make_geo(const TensorDev& d, int rb, int cb)
+{
+    Geo q;
+    const int tid = threadIdx.x;
+    const int TX = 1 << d.tx_log2;
+    q.tx = tid & (TX - 1);
+    q.ty = tid >> d.tx_log2;
+    q.TY = kThreads >> d.tx_log2;
+    q.col = (static_cast<long long>(cb) * TX + q.tx) * VEC;
+    q.colok = q.col < d.cols;
+    q.row0 = static_cast<long long>(rb) * d.tr;
+    q.row1 = min(d.rows, q.row0 + d.tr);
+    q.seg = cb * (TX >> 5) + (q.tx >> 5);
+    return q;
+}
+
+// write this tile's column partial sums (summed over the block's row groups in a fixed order)
+template <int VEC>
+__device__ __forceinline__ void write_col_partials(const TensorDev& d, const Geo& q, int rb,
+                                                   const float (&cacc)[VEC], Shared& sm)
+{
+    float out[VEC];
+    if (q.TY > 1) {
+        const int TXV = (1 << d.tx_log2) * VEC;
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) sm.colred[q.ty * TXV + q.tx * VEC + v] = cacc[v];
+        __syncthreads();
+        if (q.ty != 0) return;
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) {
+            float s = 0.f;
+            for (int y = 0; y < q.TY; ++y) s += sm.colred[y * TXV + q.tx * VEC + v];
+            out[v] = s;
+        }
+    } else {
+#pragma unroll
+        for (int v = 0; v < VEC; ++v) out[v] = cacc[v];
+    }
+    if (q.colok) store_f<VEC>(d.ws_colpart + static_cast<long long>(rb) * d.cols + q.col, out);
+}
+
+// ---------------------------------------------------------------------------
+// P1 (Algorithm 2: r_t, c_t): row and column sums of g^2
+// ---------------------------------------------------------------------------
+template <int KIND>
+__device__ __forceinline__ void p1_tile(const TensorDev& d, int rb, int cb, const StepConsts& hc,
+                                        Shared& sm)
+{
+    constexpr int VEC = Traits<KIND>::VEC;
+    constexpr int U = 8;
+    const Geo q = make_geo<VEC>(d, rb, cb);
+    const long long cols = d.cols;
+    const int lane = threadIdx.x & 31;
+    float cacc[VEC];
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) cacc[v] = 0.f;
+
+    for (long long rbase = q.row0 + q.ty; rbase < q.row1; rbase += static_cast<long long>(q.TY) * U) {
+        float x[U][VEC];
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const long long row = rbase + static_cast<long long>(k) * q.TY;
+            if (row < q.row1 && q.colok) load_g<KIND>(d.g, row * cols + q.col, x[k]);
+            else {
+#pragma unroll
+                for (int v = 0; v < VEC; ++v) x[k][v] = 0.f;
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const long long row = rbase + static_cast<long long>(k) * q.TY;
+            float rs = 0.f;
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) {
+                cacc[v] = fmaf(x[k][v], x[k][v], cacc[v]);
+                rs = fmaf(x[k][v], x[k][v], rs);
+            }
+            rs = warp_sum(rs);
+            if (lane == 0 && row < q.row1) d.ws_rowpart[q.seg * d.rows + row] = rs;
+        }
+    }
+    write_col_partials<VEC>(d, q, rb, cacc, sm);
+    finalize_factors(d, rb, cb, hc.beta2, hc.omb2, hc.eps1, 1.0f, d.r, d.c, d.scal + 0, sm);
+}
+
+// ---------------------------------------------------------------------------
+// P2 (Algorithm 2: v_t, u_t; Eq. 1): sum of u^2 -> kappa
+// ---------------------------------------------------------------------------
+template <int KIND>
+__device__ __forceinline__ void p2_tile(const TensorDev& d, int rb, int cb, const StepConsts& hc,
+                                        Shared& sm)
+{
+    constexpr int VEC = Traits<KIND>::VEC;
+    constexpr int U = 8;
+    const Geo q = make_geo<VEC>(d, rb, cb);
+    const long long cols = d.cols;
+    const float ssr = d.scal[0];
+    float b[VEC];
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) b[v] = q.colok ? __frsqrt_rn(d.c[q.col + v]) : 0.f;
+    float acc = 0.f;
+
+    for (long long rbase = q.row0 + q.ty; rbase < q.row1; rbase += static_cast<long long>(q.TY) * U) {
+        float x[U][VEC];
+        float a[U];
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const long long row = rbase + static_cast<long long>(k) * q.TY;
+            const bool ok = row < q.row1;
+            a[k] = ok ? d.r[row] : 1.f;
+            if (ok && q.colok) load_g<KIND>(d.g, row * cols + q.col, x[k]);
+            else {
+#pragma unroll
+                for (int v = 0; v < VEC; ++v) x[k][v] = 0.f;
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const float ai = __frsqrt_rn(a[k]) * ssr;
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) {
+                const float u = (x[k][v] * b[v]) * ai;
+                acc = fmaf(u, u, acc);
+            }
+        }
+    }
+    acc = block_sum(acc, sm);
+    finalize_kappa(d, rb * d.n_cb + cb, acc, hc.clip_d, sm);
+}
+
+// ---------------------------------------------------------------------------
+// P3 (Algorithm 2: uhat_t, m_t, U_t, R_t, C_t).
+// With e = uhat_t - m_{t-1}:  m_t = m_{t-1} + (1-beta1) e  and  uhat_t - m_t = beta1 e,
+// so U_t = beta1^2 e^2; the factor beta1^2 is applied once to the finished sums.
+// ---------------------------------------------------------------------------
+template <int KIND>
+__device__ __forceinline__ void p3_tile(const TensorDev& d, int rb, int cb, const StepConsts& hc,
+                                        Shared& sm)
+{
+    constexpr int VEC = Traits<KIND>::VEC;
+    constexpr int U = 4;
+    const Geo q = make_geo<VEC>(d, rb, cb);
+    const long long cols = d.cols;
+    const int lane = threadIdx.x & 31;
+    const float ssr_k = d.scal[0] * d.scal[1];          // sqrt(sum r) * kappa
+    float b[VEC], cacc[VEC];
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) {
+        b[v] = q.colok ? __frsqrt_rn(d.c[q.col + v]) : 0.f;
+        cacc[v] = 0.f;
+    }
+
+    for (long long rbase = q.row0 + q.ty; rbase < q.row1; rbase += static_cast<long long>(q.TY) * U) {
+        float x[U][VEC], mo[U][VEC], a[U];
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const long long row = rbase + static_cast<long long>(k) * q.TY;
+            const bool ok = row < q.row1;
+            a[k] = ok ? d.r[row] : 1.f;
+            if (ok && q.colok) {
+                load_g<KIND>(d.g, row * cols + q.col, x[k]);
+                load_f<VEC>(d.m + row * cols + q.col, mo[k]);
+            } else {
+#pragma unroll
+                for (int v = 0; v < VEC; ++v) { x[k][v] = 0.f; mo[k][v] = 0.f; }
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const long long row = rbase + static_cast<long long>(k) * q.TY;
+            const bool ok = row < q.row1;
+            const float ai = __frsqrt_rn(a[k]) * ssr_k;
+            float rs = 0.f;
+#pragma unroll
+            for (int v = 0; v < VEC; ++v) {
+                const float uh = (x[k][v] * b[v]) * ai;
+                const float e = uh - mo[k][v];
+                mo[k][v] = fmaf(hc.omb1, e, mo[k][v]);
+                cacc[v] = fmaf(e, e, cacc[v]);
+                rs = fmaf(e, e, rs);
+            }
+            if (ok && q.colok) store_f<VEC>(d.m + row * cols + q.col, mo[k]);
+            rs = warp_sum(rs);
+            if (lane == 0 && ok) d.ws_rowpart[q.seg * d.rows + row] = rs;
+        }
+    }
+    write_col_partials<VEC>(d, q, rb, cacc, sm);
+    finalize_factors(d, rb, cb, hc.beta3, hc.omb3, hc.eps2, hc.b1sq, d.R, d.C, d.scal + 2, sm);
+}
+
+// ---------------------------------------------------------------------------
+// P4 (Algorithm 2: S_t and the parameter line, plus decoupled decay):
+//   theta -= lr * (m * rsqrt(R_i) * sqrt(sum R) * rsqrt(C_j) + wd * theta)
+// ---------------------------------------------------------------------------
+template <int KIND>
+__device__ __forceinline__ void p4_tile(const TensorDev& d, int rb, int cb, const StepConsts& hc)
+{
+    constexpr int VEC = Traits<KIND>::VEC;
+    constexpr int U = 4;
+    const Geo q = make_geo<VEC>(d, rb, cb);
+    if (!q.colok) return;
+    const long long cols = d.cols;
+    const float ssR = d.scal[2];
+    const float wd = (d.flags & kFlagNoWd) ? 0.f : hc.wd;
+    float B[VEC];
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) B[v] = __frsqrt_rn(d.C[q.col + v]);
+
+    for (long long rbase = q.row0 + q.ty; rbase < q.row1; rbase += static_cast<long long>(q.TY) * U) {
+        float mo[U][VEC], th[U][VEC], a[U];
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const long long row = rbase + static_cast<long long>(k) * q.TY;
+            const bool ok = row < q.row1;
+            a[k] = ok ? d.R[row] : 1.f;
+            if (ok) {
+                load_f<VEC>(d.m + row * cols + q.col, mo[k]);
+                load_f<VEC>(d.p + row * cols + q.col, th[k]);
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            const long long row = rbase + static_cast<long long>(k) * q.TY;
+            if (row < q.row1) {
+                const float Ai = __frsqrt_rn(a[k]) * ssR;
+#pragma unroll
+                for (int v = 0; v < VEC; ++v) {
+                    const float upd = fmaf(wd, th[k][v], (mo[k][v] * B[v]) * Ai);
+                    th[k][v] = fmaf(-hc.lr, upd, th[k][v]);
+                }
+                store_f<VEC>(d.p + row * cols + q.col, th[k]);
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
+// kernels: one block per tile, block-uniform dispatch on the tensor's kind
+// ---------------------------------------------------------------------------
+#define CAME_DISPATCH(FN, ...)                                         \
+    switch (d.kind) {                                                  \
+        case kF32x4:  FN<kF32x4>(__VA_ARGS__);  break;                 \
+        case kBF16x8: FN<kBF16x8>(__VA_ARGS__); break;                 \
+        case kF32x1:  FN<kF32x1>(__VA_ARGS__);  break;                 \
+        default:      FN<kBF16x1>(__VA_ARGS__); break;                 \
+    }
+
+__device__ __forceinline__ Tile fetch_tile(const Tile* tiles, int ntiles, int reverse)
+{
+    const int b = static_cast<int>(blockIdx.x);
+    return tiles[reverse ? (ntiles - 1 - b) : b];
+}
+
+__global__ void __launch_bounds__(kThreads, 4)
+k_p1_reduce_g2(const TensorDev* __restrict__ T, const Tile* __restrict__ tiles, int ntiles,
+               int reverse, StepConsts hc)
+{
+    __shared__ Shared sm;
+    const Tile t = fetch_tile(tiles, ntiles, reverse);
+    const TensorDev& d = T[t.tensor];
+    CAME_DISPATCH(p1_tile, d, t.rb, t.cb, hc, sm)
+}
+
+__global__ void __launch_bounds__(kThreads, 4)
+k_p2_sum_u2(const TensorDev* __restrict__ T, const Tile* __restrict__ tiles, int ntiles,
+            int reverse, StepConsts hc)
+{
+    __shared__ Shared sm;
+    const Tile t = fetch_tile(tiles, ntiles, reverse);
+    const TensorDev& d = T[t.tensor];
+    CAME_DISPATCH(p2_tile, d, t.rb, t.cb, hc, sm)
+}
+
+__global__ void __launch_bounds__(kThreads, 2)
+k_p3_momentum_instability(const TensorDev* __restrict__ T, const Tile* __restrict__ tiles,
+                          int ntiles, int reverse, StepConsts hc)
+{
+    __shared__ Shared sm;
+    const Tile t = fetch_tile(tiles, ntiles, reverse);
+    const TensorDev& d = T[t.tensor];
+    CAME_DISPATCH(p3_tile, d, t.rb, t.cb, hc, sm)
+}
+
+__global__ void __launch_bounds__(kThreads, 2)
+k_p4_apply(const TensorDev* __restrict__ T, const Tile* __restrict__ tiles, int ntiles,
+           int reverse, StepConsts hc)
+{
+    const Tile t = fetch_tile(tiles, ntiles, reverse);
+    const TensorDev& d = T[t.tensor];
+    CAME_DISPATCH(p4_tile, d, t.rb, t.cb, hc)
+}
+
+// ---------------------------------------------------------------------------
+// vectors: the unfactored path, two kernels around the clip barrier
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ float load_grad_scalar(const TensorDev& d, long long i)
+{
+    if (d.kind == kBF16x1 || d.kind == kBF16x8)
+        return __uint_as_float(static_cast<uint32_t>(__ldg(static_cast<const uint16_t*>(d.g) + i)) << 16);
+    return __ldg(static_cast<const float*>(d.g) + i);
+}
+
+// VA: v_t = beta2 v + (1-beta2)(g^2 + eps1);  partial sums of u^2 = g^2 / v_t;  kappa
+__global__ void __launch_bounds__(kThreads)
+k_vec_second_moment(const TensorDev* __restrict__ T, const VChunk* __restrict__ chunks,
+                    StepConsts hc)
+{
+    __shared__ Shared sm;
+    const VChunk ck = chunks[blockIdx.x];
+    const TensorDev& d = T[ck.tensor];
+    const long long i0 = static_cast<long long>(ck.chunk) * kVecChunk;
+    const long long i1 = min(d.rows, i0 + kVecChunk);
+    float acc = 0.f;
+    for (long long i = i0 + threadIdx.x; i < i1; i += kThreads) {
+        const float g = load_grad_scalar(d, i);
+        const float vn = fmaf(hc.beta2, d.r[i], hc.omb2 * fmaf(g, g, hc.eps1));
+        d.r[i] = vn;
+        const float u = g * __frsqrt_rn(vn);
+        acc = fmaf(u, u, acc);
+    }
+    acc = block_sum(acc, sm);
+    finalize_kappa(d, ck.chunk, acc, hc.clip_d, sm);
+}
+
+// VB: uhat, m_t, S_t, theta_t
+__global__ void __launch_bounds__(kThreads)
+k_vec_apply(const TensorDev* __restrict__ T, const VChunk* __restrict__ chunks, StepConsts hc)
+{
+    const VChunk ck = chunks[blockIdx.x];
+    const TensorDev& d = T[ck.tensor];
+    const long long i0 = static_cast<long long>(ck.chunk) * kVecChunk;
+    const long long i1 = min(d.rows, i0 + kVecChunk);
+    const float kappa = d.scal[1];
+    const float wd = (d.flags & kFlagNoWd) ? 0.f : hc.wd;
+    const bool noconf = (d.flags & kFlagVecNoConf) != 0;
+    for (long long i = i0 + threadIdx.x; i < i1; i += kThreads) {
+        const float g = load_grad_scalar(d, i);
+        const float uh = (g * __frsqrt_rn(d.r[i])) * kappa;
+        const float mo = d.m[i];
+        const float e = uh - mo;
+        const float mn = fmaf(hc.omb1, e, mo);
+        d.m[i] = mn;
+        const float th = d.p[i];
+        float dir;
+        if (noconf) {
+            dir = mn;
+        } else {
+            const float Sn = fmaf(hc.beta3, d.R[i], hc.omb3 * fmaf(hc.b1sq * e, e, hc.eps2));
+            d.R[i] = Sn;
+            dir = mn * __frsqrt_rn(Sn);
+        }
+        d.p[i] = fmaf(-hc.lr, fmaf(wd, th, dir), th);
+    }
+}
+
+}  // namespace came
