@@ -189,6 +189,13 @@ came_status came_plan_tensor(int64_t rows, int64_t cols, int32_t ndim, int32_t g
                              int32_t* out_threads_x, int32_t* out_tile_rows, int32_t* out_n_rb,
                              int32_t* out_n_cb);
 
+/* Process-wide tuning knob, read by later came_create calls.  CAME_TUNE_TILE_ELEMS:
+ * elements per matrix tile (0 restores the default, which scales with the size
+ * of the parameter set).  Changes scheduling only, never results beyond the
+ * order of the partial sums. */
+enum { CAME_TUNE_TILE_ELEMS = 0 };
+came_status came_tune(int32_t key, int64_t value);
+
 #ifdef __cplusplus
 }
 #endif

@@ -1,0 +1,579 @@
+// Host side of the C ABI declared in include/came_b200.h: argument validation,
+// launch planning (tile list over all tensors), workspace layout, and the
+// per-step kernel launches.  All arithmetic of Algorithm 2 is in came_kernels.cuh.
+#include "../../include/came_b200.h"
+#include "came_kernels.cuh"
+
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+using came::TensorDev;
+using came::Tile;
+using came::VChunk;
+using came::StepConsts;
+
+namespace {
+
+constexpr int kMaxPhases = 6;
+const char* const kPhaseNames[kMaxPhases] = {
+    "vec_second_moment", "p1_reduce_g2", "p2_sum_u2", "p3_momentum_instability", "p4_apply",
+    "vec_apply"};
+
+thread_local std::string g_create_error;
+long long g_tile_elems_override = 0;   // came_tune(CAME_TUNE_TILE_ELEMS)
+
+struct Plan {
+    int vec = 1, tx = 256, tr = 0, n_rb = 0, n_cb = 0, n_seg = 0, n_parts = 0, kind = 0;
+};
+
+inline long long ceil_div(long long a, long long b) { return (a + b - 1) / b; }
+inline long long round_up(long long a, long long b) { return ceil_div(a, b) * b; }
+
+// Tile geometry of one tensor.  A tile is `tr` rows by `tx * vec` columns; a block of 256
+// threads covers it with tx threads across the columns and 256/tx row groups.
+Plan plan_tensor(long long rows, long long cols, int ndim, int dtype, bool aligned32,
+                 long long target)
+{
+    Plan p;
+    const bool bf = dtype == CAME_BF16;
+    if (ndim == 1) {
+        p.kind = bf ? came::kBF16x1 : came::kF32x1;
+        p.n_parts = static_cast<int>(ceil_div(rows, came::kVecChunk));
+        return p;
+    }
+    const int vmax = bf ? 8 : 4;
+    p.vec = (cols % vmax == 0 && (!bf || aligned32)) ? vmax : 1;
+    p.kind = p.vec == 1 ? (bf ? came::kBF16x1 : came::kF32x1) : (bf ? came::kBF16x8 : came::kF32x4);
+    const long long lanes = ceil_div(cols, p.vec);
+    // widest block row whose padding wastes at most 1/8 of the lanes; else the least padding
+    int best = 32;
+    long long best_pad = round_up(lanes, 32);
+    bool chosen = false;
+    for (int tx = 256; tx >= 32; tx >>= 1) {
+        const long long padded = round_up(lanes, tx);
+        if (!chosen && padded * 8 <= lanes * 9) { best = tx; chosen = true; }
+        if (!chosen && padded < best_pad) { best = tx; best_pad = padded; }
+    }
+    p.tx = best;
+    const long long sw = static_cast<long long>(p.tx) * p.vec;
+    const int ty = came::kThreads / p.tx;
+    p.n_cb = static_cast<int>(ceil_div(cols, sw));
+    if (target <= 0) target = 32768;
+    long long tr = std::max<long long>(1, target / sw);
+    tr = round_up(tr, ty);
+    tr = std::max(tr, round_up(ceil_div(rows, 256), ty));   // at most 256 row blocks per tensor
+    tr = std::min(tr, round_up(rows, ty));
+    p.tr = static_cast<int>(tr);
+    p.n_rb = static_cast<int>(ceil_div(rows, tr));
+    p.n_seg = p.n_cb * (p.tx / 32);
+    p.n_parts = p.n_rb * p.n_cb;
+    return p;
+}
+
+}  // namespace
+
+struct came_ctx {
+    int device = 0;
+    int n = 0;
+    std::vector<came_tensor> tensors;
+    std::vector<TensorDev> host_table;
+    TensorDev* d_table = nullptr;
+    TensorDev* pinned_table[2] = {nullptr, nullptr};
+    cudaEvent_t pinned_free[2] = {nullptr, nullptr};
+    bool pinned_used[2] = {false, false};
+    int pinned_next = 0;
+    Tile* d_tiles = nullptr;
+    VChunk* d_chunks = nullptr;
+    int n_tiles = 0, n_chunks = 0;
+    char* d_ws = nullptr;
+    size_t ws_bytes = 0, table_bytes = 0;
+    long long numel = 0, matrix_numel = 0, state_bytes = 0, stream_bytes = 0, comp_bytes = 0;
+    long long last_step = 0;
+    bool profiling = false;
+    cudaEvent_t ev[kMaxPhases + 1] = {};
+    int phase_of_interval[kMaxPhases] = {};
+    int n_intervals = 0;
+    bool events_valid = false;
+    std::string err;
+};
+
+namespace {
+
+came_status fail(came_ctx* ctx, came_status s, const std::string& msg)
+{
+    if (ctx) ctx->err = msg; else g_create_error = msg;
+    return s;
+}
+
+came_status cuda_fail(came_ctx* ctx, cudaError_t e, const char* what)
+{
+    std::string msg = std::string(what) + ": " + cudaGetErrorString(e);
+    const came_status s = (e == cudaErrorMemoryAllocation) ? CAME_ERR_OOM : CAME_ERR_CUDA;
+    return fail(ctx, s, msg);
+}
+
+bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+came_status validate_tensor(const came_tensor& t, int i, std::string& msg)
+{
+    char buf[160];
+    auto err = [&](came_status s, const char* what) {
+        std::snprintf(buf, sizeof buf, "tensor %d: %s", i, what);
+        msg = buf;
+        return s;
+    };
+    if (t.ndim != 1 && t.ndim != 2) return err(CAME_ERR_SHAPE, "ndim must be 1 or 2");
+    if (t.rows < 1 || t.cols < 1) return err(CAME_ERR_SHAPE, "rows and cols must be >= 1");
+    if (t.ndim == 1 && t.cols != 1) return err(CAME_ERR_SHAPE, "a vector must have cols == 1");
+    if (t.rows > (1ll << 40) / t.cols) return err(CAME_ERR_SHAPE, "tensor too large");
+    if (t.grad_dtype != CAME_F32 && t.grad_dtype != CAME_BF16) return err(CAME_ERR_DTYPE, "unknown grad_dtype");
+    if (t.reserved != 0) return err(CAME_ERR_SHAPE, "reserved must be 0");
+    if (!t.param || !t.grad || !t.m || !t.r || !t.R) return err(CAME_ERR_NULL, "param, grad, m, r, R are required");
+    if (t.ndim == 2 && (!t.c || !t.C)) return err(CAME_ERR_NULL, "a matrix needs c and C");
+    const void* ptrs[7] = {t.param, t.grad, t.m, t.r, t.c, t.R, t.C};
+    for (const void* p : ptrs)
+        if (p && !aligned(p, 16)) return err(CAME_ERR_ALIGN, "pointer not 16-byte aligned");
+    if ((t.flags & CAME_T_VEC_NO_CONFIDENCE) && t.ndim != 1)
+        return err(CAME_ERR_SHAPE, "CAME_T_VEC_NO_CONFIDENCE applies to vectors only");
+    return CAME_OK;
+}
+
+came_status validate_hparams(const came_hparams& h, long long last_step, std::string& msg)
+{
+    const double v[8] = {h.lr, h.beta1, h.beta2, h.beta3, h.eps1, h.eps2, h.clip_d, h.weight_decay};
+    for (double x : v)
+        if (!std::isfinite(x)) { msg = "hyper-parameter not finite"; return CAME_ERR_HPARAM; }
+    if (h.lr < 0) { msg = "lr must be >= 0"; return CAME_ERR_HPARAM; }
+    const double betas[3] = {h.beta1, h.beta2, h.beta3};
+    for (double b : betas)
+        if (b < 0.0 || b >= 1.0) { msg = "betas must lie in [0,1)"; return CAME_ERR_HPARAM; }
+    if (h.eps1 < 0 || h.eps2 < 0) { msg = "eps1, eps2 must be >= 0"; return CAME_ERR_HPARAM; }
+    if (!(h.clip_d > 0)) { msg = "clip_d must be > 0"; return CAME_ERR_HPARAM; }
+    if (h.weight_decay < 0) { msg = "weight_decay must be >= 0"; return CAME_ERR_HPARAM; }
+    if (h.step < 1) { msg = "step must be >= 1"; return CAME_ERR_STEP_ORDER; }
+    if (last_step > 0 && h.step != last_step + 1) {
+        msg = "step must be the previous step + 1";
+        return CAME_ERR_STEP_ORDER;
+    }
+    return CAME_OK;
+}
+
+StepConsts make_consts(const came_hparams& h)
+{
+    StepConsts c;
+    c.beta1 = static_cast<float>(h.beta1);
+    c.omb1 = static_cast<float>(1.0 - h.beta1);
+    c.b1sq = static_cast<float>(h.beta1 * h.beta1);
+    c.beta2 = static_cast<float>(h.beta2);
+    c.omb2 = static_cast<float>(1.0 - h.beta2);
+    c.beta3 = static_cast<float>(h.beta3);
+    c.omb3 = static_cast<float>(1.0 - h.beta3);
+    c.eps1 = static_cast<float>(h.eps1);
+    c.eps2 = static_cast<float>(h.eps2);
+    c.lr = static_cast<float>(h.lr);
+    c.wd = static_cast<float>(h.weight_decay);
+    c.pad_ = 0.f;
+    c.clip_d = h.clip_d;
+    return c;
+}
+
+void free_ctx(came_ctx* ctx)
+{
+    if (!ctx) return;
+    cudaSetDevice(ctx->device);
+    cudaFree(ctx->d_table);
+    cudaFree(ctx->d_tiles);
+    cudaFree(ctx->d_chunks);
+    cudaFree(ctx->d_ws);
+    for (int k = 0; k < 2; ++k) {
+        if (ctx->pinned_table[k]) cudaFreeHost(ctx->pinned_table[k]);
+        if (ctx->pinned_free[k]) cudaEventDestroy(ctx->pinned_free[k]);
+    }
+    for (cudaEvent_t e : ctx->ev)
+        if (e) cudaEventDestroy(e);
+    delete ctx;
+}
+
+// Upload the host tensor table through a pinned staging slot (two slots, each guarded by an
+// event, so that a copy still in flight from an earlier step is never overwritten).
+came_status upload_table(came_ctx* ctx, cudaStream_t stream)
+{
+    const int k = ctx->pinned_next;
+    ctx->pinned_next ^= 1;
+    if (ctx->pinned_used[k]) {
+        const cudaError_t e = cudaEventSynchronize(ctx->pinned_free[k]);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaEventSynchronize(table slot)");
+    }
+    std::memcpy(ctx->pinned_table[k], ctx->host_table.data(), ctx->table_bytes);
+    cudaError_t e = cudaMemcpyAsync(ctx->d_table, ctx->pinned_table[k], ctx->table_bytes,
+                                    cudaMemcpyHostToDevice, stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaMemcpyAsync(table)");
+    e = cudaEventRecord(ctx->pinned_free[k], stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaEventRecord(table slot)");
+    ctx->pinned_used[k] = true;
+    return CAME_OK;
+}
+
+came_status launch_step(came_ctx* ctx, const came_hparams* hp, cudaStream_t stream)
+{
+    const StepConsts hc = make_consts(*hp);
+    const bool prof = ctx->profiling;
+    int iv = 0;
+    auto mark = [&](int slot) { if (prof) cudaEventRecord(ctx->ev[slot], stream); };
+    mark(0);
+    if (ctx->n_chunks > 0) {
+        came::k_vec_second_moment<<<ctx->n_chunks, came::kThreads, 0, stream>>>(
+            ctx->d_table, ctx->d_chunks, hc);
+        ctx->phase_of_interval[iv++] = 0; mark(iv);
+    }
+    if (ctx->n_tiles > 0) {
+        came::k_p1_reduce_g2<<<ctx->n_tiles, came::kThreads, 0, stream>>>(
+            ctx->d_table, ctx->d_tiles, ctx->n_tiles, 0, hc);
+        ctx->phase_of_interval[iv++] = 1; mark(iv);
+        came::k_p2_sum_u2<<<ctx->n_tiles, came::kThreads, 0, stream>>>(
+            ctx->d_table, ctx->d_tiles, ctx->n_tiles, 1, hc);
+        ctx->phase_of_interval[iv++] = 2; mark(iv);
+        came::k_p3_momentum_instability<<<ctx->n_tiles, came::kThreads, 0, stream>>>(
+            ctx->d_table, ctx->d_tiles, ctx->n_tiles, 0, hc);
+        ctx->phase_of_interval[iv++] = 3; mark(iv);
+        came::k_p4_apply<<<ctx->n_tiles, came::kThreads, 0, stream>>>(
+            ctx->d_table, ctx->d_tiles, ctx->n_tiles, 1, hc);
+        ctx->phase_of_interval[iv++] = 4; mark(iv);
+    }
+    if (ctx->n_chunks > 0) {
+        came::k_vec_apply<<<ctx->n_chunks, came::kThreads, 0, stream>>>(
+            ctx->d_table, ctx->d_chunks, hc);
+        ctx->phase_of_interval[iv++] = 5; mark(iv);
+    }
+    ctx->n_intervals = iv;
+    ctx->events_valid = prof;
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "kernel launch");
+    ctx->last_step = hp->step;
+    return CAME_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* came_status_string(came_status s)
+{
+    switch (s) {
+        case CAME_OK: return "CAME_OK";
+        case CAME_ERR_NULL: return "CAME_ERR_NULL";
+        case CAME_ERR_SHAPE: return "CAME_ERR_SHAPE";
+        case CAME_ERR_DTYPE: return "CAME_ERR_DTYPE";
+        case CAME_ERR_ALIGN: return "CAME_ERR_ALIGN";
+        case CAME_ERR_HPARAM: return "CAME_ERR_HPARAM";
+        case CAME_ERR_STEP_ORDER: return "CAME_ERR_STEP_ORDER";
+        case CAME_ERR_DEVICE: return "CAME_ERR_DEVICE";
+        case CAME_ERR_OOM: return "CAME_ERR_OOM";
+        case CAME_ERR_CUDA: return "CAME_ERR_CUDA";
+        case CAME_ERR_INTERNAL: return "CAME_ERR_INTERNAL";
+        case CAME_ERR_UNSUPPORTED: return "CAME_ERR_UNSUPPORTED";
+    }
+    return "CAME_ERR_?";
+}
+
+const char* came_last_error(const came_ctx* ctx)
+{
+    return ctx ? ctx->err.c_str() : g_create_error.c_str();
+}
+
+came_status came_tune(int32_t key, int64_t value)
+{
+    if (key != CAME_TUNE_TILE_ELEMS || value < 0) return CAME_ERR_UNSUPPORTED;
+    g_tile_elems_override = value;
+    return CAME_OK;
+}
+
+came_status came_plan_tensor(int64_t rows, int64_t cols, int32_t ndim, int32_t grad_dtype,
+                             int32_t aligned32, int64_t tile_elems_target, int32_t* out_vec,
+                             int32_t* out_threads_x, int32_t* out_tile_rows, int32_t* out_n_rb,
+                             int32_t* out_n_cb)
+{
+    if (!out_vec || !out_threads_x || !out_tile_rows || !out_n_rb || !out_n_cb) return CAME_ERR_NULL;
+    if (rows < 1 || cols < 1 || (ndim != 1 && ndim != 2) || (ndim == 1 && cols != 1)) return CAME_ERR_SHAPE;
+    if (grad_dtype != CAME_F32 && grad_dtype != CAME_BF16) return CAME_ERR_DTYPE;
+    const Plan p = plan_tensor(rows, cols, ndim, grad_dtype, aligned32 != 0, tile_elems_target);
+    *out_vec = p.vec; *out_threads_x = p.tx; *out_tile_rows = p.tr; *out_n_rb = p.n_rb; *out_n_cb = p.n_cb;
+    return CAME_OK;
+}
+
+came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t device,
+                        uint32_t flags)
+{
+    if (!out) return fail(nullptr, CAME_ERR_NULL, "out is NULL");
+    *out = nullptr;
+    if (!t) return fail(nullptr, CAME_ERR_NULL, "tensor array is NULL");
+    if (n < 1) return fail(nullptr, CAME_ERR_SHAPE, "need at least one tensor");
+    if (flags & ~static_cast<uint32_t>(CAME_CREATE_KEEP_STATE))
+        return fail(nullptr, CAME_ERR_UNSUPPORTED, "unknown create flag");
+    std::string msg;
+    for (int i = 0; i < n; ++i) {
+        const came_status s = validate_tensor(t[i], i, msg);
+        if (s != CAME_OK) return fail(nullptr, s, msg);
+    }
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev < 1) {
+        cudaGetLastError();
+        return fail(nullptr, CAME_ERR_DEVICE, "no usable CUDA device");
+    }
+    if (device < 0 || device >= ndev) return fail(nullptr, CAME_ERR_DEVICE, "device ordinal out of range");
+    cudaError_t e = cudaSetDevice(device);
+    if (e != cudaSuccess) return cuda_fail(nullptr, e, "cudaSetDevice");
+
+    came_ctx* ctx = new (std::nothrow) came_ctx;
+    if (!ctx) return fail(nullptr, CAME_ERR_OOM, "host allocation failed");
+    ctx->device = device;
+    ctx->n = n;
+    ctx->tensors.assign(t, t + n);
+    ctx->host_table.resize(n);
+
+    // ---- plan -----------------------------------------------------------------------------
+    long long matrix_numel = 0;
+    for (int i = 0; i < n; ++i)
+        if (t[i].ndim == 2) matrix_numel += t[i].rows * t[i].cols;
+    long long target = g_tile_elems_override;
+    if (target <= 0) {
+        // aim for a few thousand tiles in all; between 4 Ki and 64 Ki elements per tile
+        target = 4096;
+        while (target < 65536 && target * 2 * 2400 <= matrix_numel) target *= 2;
+    }
+    std::vector<Plan> plans(n);
+    std::vector<Tile> tiles;
+    std::vector<VChunk> chunks;
+    size_t ws = 0;
+    auto take = [&](size_t bytes) { const size_t off = ws; ws += (bytes + 255) / 256 * 256; return off; };
+    struct Off { size_t colpart, rowpart, blocksum, usq, cnt, scal; };
+    std::vector<Off> offs(n);
+    for (int i = 0; i < n; ++i) {
+        const came_tensor& x = t[i];
+        const bool a32 = aligned(x.param, 32) && aligned(x.m, 32);
+        Plan p = plan_tensor(x.rows, x.cols, x.ndim, x.grad_dtype, a32, target);
+        plans[i] = p;
+        const long long numel = x.rows * x.cols;
+        const long long sg = x.grad_dtype == CAME_BF16 ? 2 : 4;
+        ctx->numel += numel;
+        if (x.ndim == 2) {
+            ctx->matrix_numel += numel;
+            ctx->state_bytes += 4 * (numel + 2 * (x.rows + x.cols));
+            ctx->stream_bytes += numel * (3 * sg + 20) + 16 * (x.rows + x.cols);
+            ctx->comp_bytes += numel * (sg + 16) + 16 * (x.rows + x.cols);
+            for (int rb = 0; rb < p.n_rb; ++rb)
+                for (int cb = 0; cb < p.n_cb; ++cb) tiles.push_back(Tile{i, rb, cb});
+            offs[i].colpart = take(sizeof(float) * static_cast<size_t>(p.n_rb) * x.cols);
+            offs[i].rowpart = take(sizeof(float) * static_cast<size_t>(p.n_seg) * x.rows);
+            offs[i].blocksum = take(sizeof(float) * p.n_rb);
+        } else {
+            ctx->state_bytes += 4 * 3 * numel;
+            ctx->stream_bytes += numel * (sg + 32);
+            ctx->comp_bytes += numel * (sg + 32);
+            for (int c = 0; c < p.n_parts; ++c) chunks.push_back(VChunk{i, c});
+            offs[i].colpart = offs[i].rowpart = offs[i].blocksum = 0;
+        }
+        offs[i].usq = take(sizeof(float) * p.n_parts);
+        offs[i].cnt = take(sizeof(unsigned) * (p.n_rb + p.n_cb + 2));
+        offs[i].scal = take(sizeof(float) * 4);
+        if (tiles.size() > (1u << 30) || chunks.size() > (1u << 30)) {
+            delete ctx;
+            return fail(nullptr, CAME_ERR_SHAPE, "too many tiles");
+        }
+    }
+    ctx->n_tiles = static_cast<int>(tiles.size());
+    ctx->n_chunks = static_cast<int>(chunks.size());
+    ctx->ws_bytes = ws;
+    ctx->table_bytes = sizeof(TensorDev) * n;
+
+    // ---- device memory --------------------------------------------------------------------
+#define CAME_TRY(call, what)                                                     \
+    do { e = (call); if (e != cudaSuccess) { const came_status s_ = cuda_fail(nullptr, e, what); \
+         free_ctx(ctx); return s_; } } while (0)
+    CAME_TRY(cudaMalloc(&ctx->d_ws, std::max<size_t>(ws, 256)), "cudaMalloc(workspace)");
+    CAME_TRY(cudaMemset(ctx->d_ws, 0, std::max<size_t>(ws, 256)), "cudaMemset(workspace)");
+    CAME_TRY(cudaMalloc(&ctx->d_table, ctx->table_bytes), "cudaMalloc(table)");
+    if (ctx->n_tiles) {
+        CAME_TRY(cudaMalloc(&ctx->d_tiles, sizeof(Tile) * tiles.size()), "cudaMalloc(tiles)");
+        CAME_TRY(cudaMemcpy(ctx->d_tiles, tiles.data(), sizeof(Tile) * tiles.size(),
+                            cudaMemcpyHostToDevice), "cudaMemcpy(tiles)");
+    }
+    if (ctx->n_chunks) {
+        CAME_TRY(cudaMalloc(&ctx->d_chunks, sizeof(VChunk) * chunks.size()), "cudaMalloc(chunks)");
+        CAME_TRY(cudaMemcpy(ctx->d_chunks, chunks.data(), sizeof(VChunk) * chunks.size(),
+                            cudaMemcpyHostToDevice), "cudaMemcpy(chunks)");
+    }
+    for (int k = 0; k < 2; ++k) {
+        CAME_TRY(cudaMallocHost(&ctx->pinned_table[k], ctx->table_bytes), "cudaMallocHost(table)");
+        CAME_TRY(cudaEventCreateWithFlags(&ctx->pinned_free[k], cudaEventDisableTiming), "cudaEventCreate");
+    }
+    for (cudaEvent_t& ev : ctx->ev) CAME_TRY(cudaEventCreate(&ev), "cudaEventCreate");
+
+    for (int i = 0; i < n; ++i) {
+        const came_tensor& x = t[i];
+        const Plan& p = plans[i];
+        TensorDev& d = ctx->host_table[i];
+        std::memset(&d, 0, sizeof d);
+        d.p = x.param; d.g = x.grad; d.m = x.m; d.r = x.r; d.c = x.c; d.R = x.R; d.C = x.C;
+        d.rows = x.rows; d.cols = x.cols;
+        d.ws_colpart = reinterpret_cast<float*>(ctx->d_ws + offs[i].colpart);
+        d.ws_rowpart = reinterpret_cast<float*>(ctx->d_ws + offs[i].rowpart);
+        d.ws_blocksum = reinterpret_cast<float*>(ctx->d_ws + offs[i].blocksum);
+        d.ws_usq = reinterpret_cast<float*>(ctx->d_ws + offs[i].usq);
+        d.cnt = reinterpret_cast<unsigned*>(ctx->d_ws + offs[i].cnt);
+        d.scal = reinterpret_cast<float*>(ctx->d_ws + offs[i].scal);
+        d.kind = p.kind; d.vec = p.vec;
+        int lg = 0; while ((1 << lg) < p.tx) ++lg;
+        d.tx_log2 = lg; d.tr = p.tr; d.n_rb = p.n_rb; d.n_cb = p.n_cb; d.n_seg = p.n_seg;
+        d.n_parts = p.n_parts; d.ndim = x.ndim; d.flags = x.flags;
+        if (!(flags & CAME_CREATE_KEEP_STATE)) {
+            const size_t numel = static_cast<size_t>(x.rows) * x.cols;
+            CAME_TRY(cudaMemsetAsync(x.m, 0, 4 * numel, 0), "cudaMemset(m)");
+            CAME_TRY(cudaMemsetAsync(x.r, 0, 4 * static_cast<size_t>(x.rows), 0), "cudaMemset(r)");
+            CAME_TRY(cudaMemsetAsync(x.R, 0, 4 * static_cast<size_t>(x.rows), 0), "cudaMemset(R)");
+            if (x.ndim == 2) {
+                CAME_TRY(cudaMemsetAsync(x.c, 0, 4 * static_cast<size_t>(x.cols), 0), "cudaMemset(c)");
+                CAME_TRY(cudaMemsetAsync(x.C, 0, 4 * static_cast<size_t>(x.cols), 0), "cudaMemset(C)");
+            }
+        }
+    }
+    CAME_TRY(cudaMemcpy(ctx->d_table, ctx->host_table.data(), ctx->table_bytes,
+                        cudaMemcpyHostToDevice), "cudaMemcpy(table)");
+    CAME_TRY(cudaDeviceSynchronize(), "cudaDeviceSynchronize");
+#undef CAME_TRY
+    *out = ctx;
+    return CAME_OK;
+}
+
+came_status came_step(came_ctx* ctx, const came_hparams* hp, const void* const* grads,
+                      void* cuda_stream)
+{
+    if (!ctx) return CAME_ERR_NULL;
+    if (!hp) return fail(ctx, CAME_ERR_NULL, "hparams is NULL");
+    std::string msg;
+    came_status s = validate_hparams(*hp, ctx->last_step, msg);
+    if (s != CAME_OK) return fail(ctx, s, msg);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    if (grads) {
+        bool changed = false;
+        for (int i = 0; i < ctx->n; ++i) {
+            if (!grads[i]) return fail(ctx, CAME_ERR_NULL, "a gradient pointer is NULL");
+            if (!aligned(grads[i], 16)) return fail(ctx, CAME_ERR_ALIGN, "gradient pointer not 16-byte aligned");
+            changed |= (grads[i] != ctx->host_table[i].g);
+        }
+        if (changed) {
+            for (int i = 0; i < ctx->n; ++i) { ctx->host_table[i].g = grads[i]; ctx->tensors[i].grad = grads[i]; }
+            s = upload_table(ctx, stream);
+            if (s != CAME_OK) return s;
+        }
+    }
+    return launch_step(ctx, hp, stream);
+}
+
+came_status came_step_host(came_ctx* ctx, const came_hparams* hp, const void* const* host_grads,
+                           void* const* host_params_out, void* cuda_stream)
+{
+    if (!ctx) return CAME_ERR_NULL;
+    if (!hp || !host_grads) return fail(ctx, CAME_ERR_NULL, "hparams or host_grads is NULL");
+    std::string msg;
+    came_status s = validate_hparams(*hp, ctx->last_step, msg);
+    if (s != CAME_OK) return fail(ctx, s, msg);
+    for (int i = 0; i < ctx->n; ++i)
+        if (!host_grads[i]) return fail(ctx, CAME_ERR_NULL, "a host gradient pointer is NULL");
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    for (int i = 0; i < ctx->n; ++i) {
+        const came_tensor& x = ctx->tensors[i];
+        const size_t bytes = static_cast<size_t>(x.rows) * x.cols * (x.grad_dtype == CAME_BF16 ? 2 : 4);
+        const cudaError_t e = cudaMemcpyAsync(const_cast<void*>(x.grad), host_grads[i], bytes,
+                                              cudaMemcpyHostToDevice, stream);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaMemcpyAsync(grad H2D)");
+    }
+    s = launch_step(ctx, hp, stream);
+    if (s != CAME_OK) return s;
+    if (host_params_out) {
+        for (int i = 0; i < ctx->n; ++i) {
+            if (!host_params_out[i]) continue;
+            const came_tensor& x = ctx->tensors[i];
+            const size_t bytes = static_cast<size_t>(x.rows) * x.cols * 4;
+            const cudaError_t e = cudaMemcpyAsync(host_params_out[i], x.param, bytes,
+                                                  cudaMemcpyDeviceToHost, stream);
+            if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaMemcpyAsync(param D2H)");
+        }
+    }
+    return CAME_OK;
+}
+
+came_status came_destroy(came_ctx* ctx)
+{
+    if (!ctx) return CAME_ERR_NULL;
+    free_ctx(ctx);
+    return CAME_OK;
+}
+
+came_status came_query(const came_ctx* ctx, int32_t what, int64_t* out)
+{
+    if (!ctx || !out) return CAME_ERR_NULL;
+    switch (what) {
+        case CAME_Q_NUMEL: *out = ctx->numel; break;
+        case CAME_Q_STATE_BYTES: *out = ctx->state_bytes; break;
+        case CAME_Q_STREAM_BYTES: *out = ctx->stream_bytes; break;
+        case CAME_Q_COMPULSORY_BYTES: *out = ctx->comp_bytes; break;
+        case CAME_Q_WORKSPACE_BYTES:
+            *out = static_cast<int64_t>(ctx->ws_bytes + ctx->table_bytes + sizeof(Tile) * ctx->n_tiles +
+                                        sizeof(VChunk) * ctx->n_chunks);
+            break;
+        case CAME_Q_NUM_TILES: *out = ctx->n_tiles; break;
+        case CAME_Q_LAUNCHES_PER_STEP: *out = (ctx->n_tiles ? 4 : 0) + (ctx->n_chunks ? 2 : 0); break;
+        case CAME_Q_LAST_STEP: *out = ctx->last_step; break;
+        case CAME_Q_NUM_PHASES: *out = (ctx->n_tiles ? 4 : 0) + (ctx->n_chunks ? 2 : 0); break;
+        case CAME_Q_MATRIX_NUMEL: *out = ctx->matrix_numel; break;
+        default: return CAME_ERR_UNSUPPORTED;
+    }
+    return CAME_OK;
+}
+
+came_status came_set_profiling(came_ctx* ctx, int32_t enabled)
+{
+    if (!ctx) return CAME_ERR_NULL;
+    ctx->profiling = enabled != 0;
+    ctx->events_valid = false;
+    return CAME_OK;
+}
+
+came_status came_get_phase_ms(came_ctx* ctx, float* out_ms, int32_t cap, int32_t* out_count)
+{
+    if (!ctx || !out_ms || !out_count) return CAME_ERR_NULL;
+    *out_count = 0;
+    if (!ctx->events_valid) return fail(ctx, CAME_ERR_UNSUPPORTED, "no profiled step recorded");
+    cudaError_t e = cudaEventSynchronize(ctx->ev[ctx->n_intervals]);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaEventSynchronize");
+    const int k = std::min<int>(cap, ctx->n_intervals);
+    for (int i = 0; i < k; ++i) {
+        e = cudaEventElapsedTime(&out_ms[i], ctx->ev[i], ctx->ev[i + 1]);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaEventElapsedTime");
+    }
+    *out_count = k;
+    return CAME_OK;
+}
+
+const char* came_phase_name(const came_ctx* ctx, int32_t phase)
+{
+    if (!ctx || phase < 0) return "";
+    // phases are reported in launch order; vectors-only or matrices-only contexts skip some
+    int idx = 0;
+    const bool has[kMaxPhases] = {ctx->n_chunks > 0, ctx->n_tiles > 0, ctx->n_tiles > 0,
+                                  ctx->n_tiles > 0, ctx->n_tiles > 0, ctx->n_chunks > 0};
+    for (int k = 0; k < kMaxPhases; ++k) {
+        if (!has[k]) continue;
+        if (idx == phase) return kPhaseNames[k];
+        ++idx;
+    }
+    return "";
+}
+
+}  // extern "C"
