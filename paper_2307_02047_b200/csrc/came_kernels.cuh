@@ -537,7 +537,7 @@ __device__ __forceinline__ Tile fetch_tile(const Tile* tiles, int ntiles, int re
     return tiles[reverse ? (ntiles - 1 - b) : b];
 }
 
-__global__ void __launch_bounds__(kThreads, 3)
+__global__ void __launch_bounds__(kThreads, 2)
 k_p1_reduce_g2(const TensorDev* __restrict__ T, const Tile* __restrict__ tiles, int ntiles,
                int reverse, StepConsts hc)
 {
@@ -547,7 +547,7 @@ k_p1_reduce_g2(const TensorDev* __restrict__ T, const Tile* __restrict__ tiles, 
     CAME_DISPATCH(p1_tile, d, t.rb, t.cb, hc, sm)
 }
 
-__global__ void __launch_bounds__(kThreads, 3)
+__global__ void __launch_bounds__(kThreads, 2)
 k_p2_sum_u2(const TensorDev* __restrict__ T, const Tile* __restrict__ tiles, int ntiles,
             int reverse, StepConsts hc)
 {

@@ -1,0 +1,76 @@
+"""Shared helpers for the GPU parity tests: error measures and a paired runner that
+feeds identical seeded inputs to the CUDA library (through its C ABI) and to the
+CPU float64 oracle."""
+from __future__ import annotations
+
+import numpy as np
+
+from paper_2307_02047_b200 import synth
+
+# Tolerances: max error <= 1e-5 after one step and <= 1e-4 after ten steps (fp32 state).
+TOL_STEP1 = 1e-5
+TOL_STEP10 = 1e-4
+
+
+def err_signed(x: np.ndarray, ref: np.ndarray) -> float:
+    """For p and m (signed, cancelling): max |x - ref| / (|ref| + RMS(ref))."""
+    ref = ref.astype(np.float64)
+    rms = float(np.sqrt(np.mean(ref * ref)))
+    den = np.abs(ref) + rms
+    den[den == 0.0] = 1.0
+    return float(np.max(np.abs(x.astype(np.float64) - ref) / den))
+
+
+def err_positive(x: np.ndarray, ref: np.ndarray) -> float:
+    """For the positive reductions r, c, R, C (and vector v, S): strict element-wise relative error."""
+    ref = ref.astype(np.float64)
+    return float(np.max(np.abs(x.astype(np.float64) - ref) / ref))
+
+
+def to_torch_grad(torch, g: np.ndarray, device):
+    if g.dtype == np.uint16:
+        return torch.from_numpy(g.view(np.int16)).view(torch.bfloat16).to(device)
+    return torch.from_numpy(g).to(device)
+
+
+def compare_state(opt, orc, indices=None) -> dict:
+    """Worst error per state name between a CameOptimizer and an OracleOptimizer."""
+    worst = dict(p=0.0, m=0.0, r=0.0, c=0.0, R=0.0, C=0.0)
+    idx = range(len(opt.params)) if indices is None else indices
+    for k, i in enumerate(idx):
+        j = i if indices is None else k
+        worst["p"] = max(worst["p"], err_signed(opt.params[i].cpu().numpy(), orc.p[j]))
+        worst["m"] = max(worst["m"], err_signed(opt.m[i].cpu().numpy(), orc.m[j]))
+        worst["r"] = max(worst["r"], err_positive(opt.r[i].cpu().numpy(), orc.r[j]))
+        worst["R"] = max(worst["R"], err_positive(opt.R[i].cpu().numpy(), orc.R[j]))
+        if opt.c[i] is not None:
+            worst["c"] = max(worst["c"], err_positive(opt.c[i].cpu().numpy(), orc.c[j]))
+            worst["C"] = max(worst["C"], err_positive(opt.C[i].cpu().numpy(), orc.C[j]))
+    return worst
+
+
+def run_paired(torch, binding, oracle, w: synth.Workload, seed: int, steps: int, check_at,
+               flags=None, hparams=None, device="cuda:0"):
+    """Step the CUDA path and the oracle side by side; returns {step: worst-error dict}."""
+    hp = dict(w.hparams if hparams is None else hparams)
+    params = synth.make_params(w, seed)
+    dev_p = [torch.from_numpy(p.copy()).to(device) for p in params]
+    g0 = synth.make_grads(w, seed, 1)
+    dev_g = [to_torch_grad(torch, g, device) for g in g0]
+    opt = binding.CameOptimizer(dev_p, dev_g, flags=flags)
+    no_wd = [bool(f & binding.CAME_T_NO_WEIGHT_DECAY) for f in flags] if flags else ()
+    no_conf = [bool(f & binding.CAME_T_VEC_NO_CONFIDENCE) for f in flags] if flags else ()
+    orc = oracle.OracleOptimizer(params, no_weight_decay=no_wd, vec_no_confidence=no_conf)
+    out = {}
+    for step in range(1, steps + 1):
+        grads = g0 if step == 1 else synth.make_grads(w, seed, step)
+        if step > 1:
+            for dg, g in zip(dev_g, grads):
+                dg.copy_(to_torch_grad(torch, g, device))
+        opt.step(**hp)
+        orc.step([synth.widen(g) for g in grads], **hp)
+        if step in check_at:
+            torch.cuda.synchronize()
+            out[step] = compare_state(opt, orc)
+    opt.close()
+    return out

@@ -1,0 +1,122 @@
+"""CPU-only checks of the C-ABI library: it loads, exports every symbol the header declares,
+rejects bad arguments before touching CUDA, and its host-side tile planner covers every
+matrix exactly once.  No GPU compute is called here."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2307_02047_b200 import binding, synth
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_functions():
+    text = open(os.path.join(ROOT, "include", "came_b200.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(came_[a-z_]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported():
+    L = binding.load()
+    names = _declared_functions()
+    assert len(names) >= 10
+    for n in names:
+        assert hasattr(L, n), f"{n} declared in the header but not exported"
+    assert sorted(binding.EXPORTED) == names
+
+
+def _desc(rows=8, cols=8, ndim=2, dt=0, base=0x10000, flags=0, **over):
+    d = dict(param=base, grad=base + 0x1000, m=base + 0x2000, r=base + 0x3000,
+             c=(base + 0x4000) if ndim == 2 else None, R=base + 0x5000,
+             C=(base + 0x6000) if ndim == 2 else None)
+    d.update(over)
+    return binding.came_tensor(d["param"], d["grad"], d["m"], d["r"], d["c"], d["R"], d["C"],
+                               rows, cols, ndim, dt, flags, 0)
+
+
+@pytest.mark.parametrize("desc,status", [
+    (dict(ndim=3), 2), (dict(rows=0), 2), (dict(cols=0), 2), (dict(ndim=1, cols=4), 2),
+    (dict(dt=7), 3), (dict(param=None), 1), (dict(c=None), 1), (dict(C=None), 1),
+    (dict(m=0x10008), 4), (dict(grad=0x10002), 4), (dict(flags=2), 2),
+])
+def test_create_rejects_bad_descriptors_without_cuda(desc, status):
+    with pytest.raises(binding.CameError) as e:
+        binding.came_create([_desc(**desc)])
+    assert e.value.status == status
+    assert binding.came_last_error(None) != ""
+
+
+def test_create_null_and_count():
+    L = binding.load()
+    ctx = ctypes.c_void_p()
+    assert L.came_create(None, None, 1, 0, 0) == 1
+    assert L.came_create(ctypes.byref(ctx), None, 1, 0, 0) == 1
+    arr = (binding.came_tensor * 1)(_desc())
+    assert L.came_create(ctypes.byref(ctx), arr, 0, 0, 0) == 2
+    assert L.came_create(ctypes.byref(ctx), arr, 1, 0, 0xF0) == 11
+    assert ctx.value is None
+    assert L.came_step(None, None, None, None) == 1
+    assert L.came_destroy(None) == 1
+    assert binding.came_status_string(5) == "CAME_ERR_HPARAM"
+
+
+def test_create_without_gpu_reports_device_error():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    with pytest.raises(binding.CameError) as e:
+        binding.came_create([_desc()])
+    assert e.value.status == 7      # CAME_ERR_DEVICE: no silent CPU fallback
+
+
+SHAPES = [(1, 1), (1, 65536), (65536, 1), (30522, 768), (768, 3072), (3072, 768), (4096, 11008),
+          (11008, 4096), (128256, 4096), (16384, 16384), (513, 1030), (50257, 1024), (7, 13)]
+
+
+@pytest.mark.parametrize("dt", [0, 1])
+@pytest.mark.parametrize("target", [0, 4096, 65536])
+@pytest.mark.parametrize("shape", SHAPES)
+def test_plan_covers_matrix_exactly(shape, dt, target):
+    rows, cols = shape
+    p = binding.came_plan_tensor(rows, cols, 2, dt, True, target)
+    vec, tx, tr = p["vec"], p["threads_x"], p["tile_rows"]
+    assert vec in (1, 4, 8) and tx in (32, 64, 128, 256)
+    assert cols % vec == 0
+    sw = tx * vec
+    ty = 256 // tx
+    assert tr >= 1 and tr % ty == 0
+    # row blocks and column strips tile the matrix with no gap and no overlap
+    assert (p["n_rb"] - 1) * tr < rows <= p["n_rb"] * tr
+    assert (p["n_cb"] - 1) * sw < cols <= p["n_cb"] * sw
+    assert p["n_rb"] <= 256 or tr >= rows // 256
+    if vec > 1:
+        assert (vec == 8) == (dt == 1)
+
+
+def test_plan_unaligned_bf16_falls_back_to_scalar():
+    assert binding.came_plan_tensor(64, 1024, 2, 1, False, 0)["vec"] == 1
+    assert binding.came_plan_tensor(64, 1024, 2, 0, False, 0)["vec"] == 4
+    assert binding.came_plan_tensor(64, 1022, 2, 0, True, 0)["vec"] == 1
+
+
+def test_plan_rejects_bad_arguments():
+    L = binding.load()
+    o = [ctypes.c_int32() for _ in range(5)]
+    refs = [ctypes.byref(x) for x in o]
+    assert L.came_plan_tensor(0, 4, 2, 0, 1, 0, *refs) == 2
+    assert L.came_plan_tensor(4, 4, 2, 9, 1, 0, *refs) == 3
+    assert L.came_plan_tensor(4, 4, 2, 0, 1, 0, None, *refs[1:]) == 1
+    assert L.came_tune(99, 1) == 11
+
+
+def test_workload_shapes_match_the_named_models():
+    counts = {"toy": (1, 1, 512 * 256 + 256), "bert_base": (74, 120, 108_888_576),
+              "bert_large": (146, 240, 334_088_192), "gpt2_medium": (98, 192, 354_821_120),
+              "llama7b": (226, 65, 6_738_415_616)}
+    for name, (nm, nv, numel) in counts.items():
+        w = synth.workload(name)
+        assert sum(t.ndim == 2 for t in w.tensors) == nm
+        assert sum(t.ndim == 1 for t in w.tensors) == nv
+        assert w.numel == numel

@@ -1,0 +1,92 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU float64 oracle
+on identical seeded inputs.  Gates: 1e-5 after one step, 1e-4 after ten steps."""
+import numpy as np
+import pytest
+
+from paper_2307_02047_b200 import synth
+from tests.parity_util import TOL_STEP1, TOL_STEP10, run_paired
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def env(oracle):
+    import torch
+    from paper_2307_02047_b200 import binding
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    binding.load()
+    return torch, binding, oracle
+
+
+def _gate(res):
+    for step, worst in res.items():
+        tol = TOL_STEP1 if step == 1 else TOL_STEP10
+        for name, e in worst.items():
+            assert e <= tol, f"step {step}: {name} error {e:.3e} > {tol:.0e}  ({worst})"
+
+
+def test_toy_config_ten_steps(env):
+    torch, binding, oracle = env
+    _gate(run_paired(torch, binding, oracle, synth.workload("toy"), seed=1, steps=10, check_at=(1, 10)))
+
+
+SHAPES = [(1, 1), (1, 37), (37, 1), (5, 3), (33, 65), (64, 256), (257, 1030), (1000, 72),
+          (300, 2052), (2, 4096), (1, 65536), (65536, 1), (777, 768), (513, 3072)]
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("shape", SHAPES)
+def test_single_matrix_shapes(env, shape, dtype):
+    torch, binding, oracle = env
+    w = synth.workload(f"mat:{shape[0]}x{shape[1]}" + (":bf16" if dtype == "bf16" else ""))
+    _gate(run_paired(torch, binding, oracle, w, seed=3, steps=3, check_at=(1, 3)))
+
+
+@pytest.mark.parametrize("tile", [4096, 8192, 65536])
+def test_tile_sizes_span_many_tiles(env, tile):
+    torch, binding, oracle = env
+    binding.came_tune(binding.CAME_TUNE_TILE_ELEMS, tile)
+    try:
+        w = synth.workload("mat:1500x1288:bf16")
+        _gate(run_paired(torch, binding, oracle, w, seed=5, steps=10, check_at=(1, 10)))
+    finally:
+        binding.came_tune(binding.CAME_TUNE_TILE_ELEMS, 0)
+
+
+@pytest.mark.parametrize("n", [1, 7, 256, 4097, 100003])
+def test_vectors(env, n):
+    torch, binding, oracle = env
+    w = synth.Workload("v", (synth.vec("b", n),), synth.F32, "normal_fixed", 1e-3, 0.0, (), 3,
+                       dict(synth.PAPER_HPARAMS))
+    _gate(run_paired(torch, binding, oracle, w, seed=7, steps=3, check_at=(1, 3)))
+
+
+def test_flags_weight_decay_and_no_confidence(env):
+    torch, binding, oracle = env
+    ts = (synth.mat("w0", 130, 264), synth.mat("w1", 64, 128), synth.vec("b0", 300), synth.vec("b1", 300))
+    hp = dict(synth.PAPER_HPARAMS, weight_decay=0.01)
+    w = synth.Workload("flags", ts, synth.BF16, "student_t3", 1e-3, 0.0, (), 10, hp)
+    flags = [0, binding.CAME_T_NO_WEIGHT_DECAY, binding.CAME_T_VEC_NO_CONFIDENCE,
+             binding.CAME_T_NO_WEIGHT_DECAY]
+    _gate(run_paired(torch, binding, oracle, w, seed=9, steps=10, check_at=(1, 10), flags=flags))
+
+
+def test_zero_rows_everywhere(env):
+    torch, binding, oracle = env
+    ts = (synth.mat("e", 3000, 256), synth.mat("w", 256, 1024), synth.vec("b", 256))
+    w = synth.Workload("z", ts, synth.BF16, "normal_loguniform", 0.0, 0.0, (), 10,
+                       dict(synth.PAPER_HPARAMS))
+    w = synth.with_zero_rows_everywhere(w, 0.2)
+    res = run_paired(torch, binding, oracle, w, seed=11, steps=10, check_at=(1, 10))
+    _gate(res)
+
+
+def test_other_hyperparameters(env):
+    torch, binding, oracle = env
+    hp = dict(lr=1e-3, beta1=0.8, beta2=0.99, beta3=0.999, eps1=1e-12, eps2=1e-6, clip_d=0.5,
+              weight_decay=0.1)
+    _gate(run_paired(torch, binding, oracle, synth.workload("toy"), seed=13, steps=10,
+                     check_at=(1, 10), hparams=hp))
+    hp0 = dict(synth.PAPER_HPARAMS, beta1=0.0, clip_d=100.0)
+    _gate(run_paired(torch, binding, oracle, synth.workload("toy"), seed=13, steps=3,
+                     check_at=(1, 3), hparams=hp0))
