@@ -1,0 +1,391 @@
+#!/usr/bin/env python
+"""Benchmark of the CAME optimizer step (Algorithm 2) on B200.
+
+One "step" is one full came_step over the whole parameter set: all four matrix phases
+plus the vector kernels.  Default workload: the LLaMA-7B-shaped set (6.74 B fp32
+parameters, bf16 gradients), the largest single-GPU configuration.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+Prints ONE JSON line (rank 0).  With N > 1 (launched by torchrun) every rank runs an
+independent replica of the workload on its own GPU -- the path has no exchange step, so
+there is no collective in the data path -- and the time is the max over ranks.
+--impl reference times the CPU float64 oracle instead, on a bounded sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2307_02047_b200 import synth  # noqa: E402
+
+METRIC = "came_params_updated_per_sec"
+UNIT = "params/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+def dist_env():
+    return int(os.environ.get("RANK", 0)), int(os.environ.get("LOCAL_RANK", 0)), \
+        int(os.environ.get("WORLD_SIZE", 1))
+
+
+# ---------------------------------------------------------------------------------------
+# clocks
+# ---------------------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.path = tempfile.mktemp(prefix="came_clocks_", suffix=".csv")
+        self.proc = None
+        self.idx = gpu_index
+
+    def start(self):
+        try:
+            self.f = open(self.path, "w")
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.idx), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.f.close()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        try:
+            for line in open(self.path):
+                parts = [x.strip() for x in line.split(",")]
+                if len(parts) < 7:
+                    continue
+                try:
+                    sm.append(float(parts[0])); mx.append(float(parts[1]))
+                except ValueError:
+                    continue
+                for n, v in zip(names, parts[3:7]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+            os.unlink(self.path)
+        except Exception:
+            pass
+        if sm:
+            sm.sort()
+            out.update(sm_mhz=sm[len(sm) // 2], sm_max_mhz=max(mx), samples=len(sm))
+        out["reasons"] = sorted(reasons)
+        return out
+
+
+# ---------------------------------------------------------------------------------------
+# GPU arm
+# ---------------------------------------------------------------------------------------
+def alloc_device_workload(torch, w: synth.Workload, device):
+    gen = torch.Generator(device=device)
+    gen.manual_seed(1234)
+    params, grads = [], []
+    gdt = torch.bfloat16 if w.grad_dtype == synth.BF16 else torch.float32
+    for t in w.tensors:
+        p = torch.empty(t.shape, dtype=torch.float32, device=device)
+        p.normal_(0.0, 0.02, generator=gen)
+        g = torch.empty(t.shape, dtype=gdt, device=device)
+        g.normal_(0.0, 1e-3, generator=gen)
+        params.append(p)
+        grads.append(g)
+    return params, grads
+
+
+def phase_bytes(w: synth.Workload):
+    """Algorithmic bytes per launch of each matrix phase (matrix elements only + factors)."""
+    sg = 2 if w.grad_dtype == synth.BF16 else 4
+    nm = sum(t.numel for t in w.tensors if t.ndim == 2)
+    fac = sum(t.rows + t.cols for t in w.tensors if t.ndim == 2)
+    return {"p1_reduce_g2": nm * sg + 8 * fac, "p2_sum_u2": nm * sg + 4 * fac,
+            "p3_momentum_instability": nm * (sg + 8) + 12 * fac, "p4_apply": nm * 12 + 4 * fac}
+
+
+def run_gpu(args):
+    import torch
+    from paper_2307_02047_b200 import binding
+    rank, local_rank, world = dist_env()
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    binding.load()                      # raises if the CUDA library cannot be had: no fallback
+    w = synth.workload(args.workload)
+    hp = dict(w.hparams)
+    params, grads = alloc_device_workload(torch, w, device)
+    opt = binding.CameOptimizer(params, grads, device=local_rank)
+    numel = opt.query(binding.CAME_Q_NUMEL)
+    stream_bytes = opt.query(binding.CAME_Q_STREAM_BYTES)
+    launches = opt.query(binding.CAME_Q_LAUNCHES_PER_STEP)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        opt.step(**hp)
+    barrier()
+    binding.came_set_profiling(opt.ctx, True)
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(args.steps):
+        opt.step(**hp)
+    ev1.record()
+    barrier()
+    ms = ev0.elapsed_time(ev1)
+    clocks = sampler.stop() if rank == 0 else {}
+    phase_ms = binding.came_get_phase_ms(opt.ctx)
+    phase_names = [binding.came_phase_name(opt.ctx, i) for i in range(len(phase_ms))]
+    binding.came_set_profiling(opt.ctx, False)
+    if world > 1:
+        t = torch.tensor([ms], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms_per_step = ms / args.steps
+    value = world * numel / (ms_per_step * 1e-3)
+
+    # ---- end to end: host gradients in, updated parameters out, every step --------------
+    e2e = run_e2e(torch, binding, opt, w, hp, device, world, rank, args)
+
+    peak, peak_kind = measured_peak()
+    pb = phase_bytes(w)
+    phases = {n: m for n, m in zip(phase_names, phase_ms)}
+    matrix_phases = {n: m for n, m in phases.items() if n in pb}
+    roofline = None
+    if matrix_phases:
+        dom = max(matrix_phases, key=matrix_phases.get)
+        ach = pb[dom] / (matrix_phases[dom] * 1e-3) / 1e9
+        roofline = {"bound": "hbm", "kernel": dom, "achieved": round(ach, 1), "peak": peak,
+                    "peak_kind": peak_kind, "unit": "GB/s", "frac": round(ach / peak, 4),
+                    "traffic": TRAFFIC_BYTES.get((args.workload, dom)),
+                    "algorithmic_bytes_per_launch": pb[dom],
+                    "per_phase": {n: {"ms": round(m, 4), "GB/s": round(pb[n] / (m * 1e-3) / 1e9, 1)}
+                                  for n, m in matrix_phases.items()}}
+    eff_gbs = stream_bytes / (ms_per_step * 1e-3) / 1e9
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": args.workload, "params": numel,
+                   "tensors": len(w.tensors), "grad_dtype": w.grad_dtype,
+                   "state": "fp32 params, m, r, c, R, C",
+                   "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "l2": "per-step working set %.1f GB >> 126 MB L2; no flush needed"
+                         % (stream_bytes / 1e9) if stream_bytes > 1e9 else
+                         "working set comparable to L2: L2-resident, not an HBM measurement"},
+        "hbm": {"stream_bytes_per_step": stream_bytes, "effective_GBps": round(eff_gbs, 1),
+                "frac_of_nominal_8TBps": round(eff_gbs / NOMINAL_HBM_GBS, 4),
+                "frac_of_%s_%.1f" % (peak_kind, peak): round(eff_gbs / peak, 4)},
+        "clocks": clocks, "e2e": e2e, "gpu_launches": launches * args.steps,
+        "roofline": roofline,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        line["cpu_baseline"] = cpu_baseline(budget_s=25.0, steps=1, warmup=0)
+    opt.close()
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+
+
+# ncu-measured DRAM bytes per launch of the dominant kernel (read + write), keyed by
+# (workload, kernel).  None until a capture of the current kernel exists.
+TRAFFIC_BYTES = {}
+
+
+def host_mem_available() -> int:
+    try:
+        for line in open("/proc/meminfo"):
+            if line.startswith("MemAvailable:"):
+                return int(line.split()[1]) * 1024
+    except Exception:
+        pass
+    return 0
+
+
+def run_e2e(torch, binding, opt, w, hp, device, world, rank, args):
+    """Same step through came_step_host: pinned host gradients -> device, step, parameters -> host."""
+    sg = 2 if w.grad_dtype == synth.BF16 else 4
+    h2d = sum(t.numel for t in w.tensors) * sg
+    d2h = sum(t.numel for t in w.tensors) * 4
+    need = h2d + d2h
+    budget = host_mem_available() // (2 * max(world, 1))
+    shared = need > budget
+    gdt = torch.bfloat16 if w.grad_dtype == synth.BF16 else torch.float32
+    hg, hp_out = [], []
+    pool_g, pool_p = {}, {}
+    for t, g in zip(w.tensors, opt.grads):
+        if shared:       # not enough host memory for one buffer per tensor: one per distinct shape
+            if t.shape not in pool_g:
+                pool_g[t.shape] = torch.empty(t.shape, dtype=gdt).pin_memory()
+                pool_g[t.shape].copy_(g)
+                pool_p[t.shape] = torch.empty(t.shape, dtype=torch.float32).pin_memory()
+            hg.append(pool_g[t.shape]); hp_out.append(pool_p[t.shape])
+        else:
+            b = torch.empty(t.shape, dtype=gdt).pin_memory()
+            b.copy_(g)
+            hg.append(b)
+            hp_out.append(torch.empty(t.shape, dtype=torch.float32).pin_memory())
+    gptr = [x.data_ptr() for x in hg]
+    pptr = [x.data_ptr() for x in hp_out]
+    stream = torch.cuda.current_stream().cuda_stream
+    steps = max(1, min(args.steps, args.e2e_steps))
+
+    def one():
+        opt.step_count += 1
+        binding.came_step_host(opt.ctx, binding.make_hparams(opt.step_count, **hp), gptr, pptr, stream)
+
+    one()
+    torch.cuda.synchronize()
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for _ in range(steps):
+        one()
+    ev1.record()
+    torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1) / steps
+    if world > 1:
+        tt = torch.tensor([ms], device=device)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms = float(tt.item())
+    numel = sum(t.numel for t in w.tensors)
+    return {"value": world * numel / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms, "steps": steps,
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+            "api": "came_step_host (pinned host gradients in, updated fp32 parameters out)",
+            "host_buffers": "one pinned buffer per distinct shape (host memory budget)" if shared
+                            else "one pinned buffer per tensor"}
+
+
+# ---------------------------------------------------------------------------------------
+# CPU oracle arm
+# ---------------------------------------------------------------------------------------
+def _oracle_sample(budget_s: float, total_steps: int):
+    """Pick the bounded sample of the LLaMA-7B-shaped set the oracle is timed on."""
+    import numpy as np
+    from oracle import came_oracle
+    came_oracle.build()
+    # calibrate on one 1024 x 4096 matrix (4.2 M elements)
+    cal = synth.Workload("cal", (synth.mat("w", 1024, 4096),), synth.BF16, "normal_fixed", 1e-3,
+                         0.0, (), 1, dict(synth.PAPER_HPARAMS))
+    p = synth.make_params(cal, 1)
+    o = came_oracle.OracleOptimizer(p)
+    g = [synth.widen(x) for x in synth.make_grads(cal, 1, 1)]
+    o.step(g, **cal.hparams)
+    t0 = time.perf_counter()
+    o.step(g, **cal.hparams)
+    per_elem = (time.perf_counter() - t0) / cal.numel
+    layer = synth.workload("llama7b_layer")
+    if per_elem * layer.numel * total_steps <= budget_s:
+        return layer, "one transformer layer of the LLaMA-7B-shaped set (7 matrices + 2 vectors, 202.4 M parameters)"
+    small = synth.Workload("llama7b_slice", (synth.mat("wq", 4096, 4096), synth.mat("w_gate", 4096, 11008),
+                                             synth.vec("norm1", 4096)), synth.BF16, "normal_fixed",
+                           1e-3, 0.0, (), 1, dict(synth.PAPER_HPARAMS))
+    if per_elem * small.numel * total_steps <= budget_s:
+        return small, "one 4096x4096 and one 4096x11008 matrix plus one 4096 vector of the LLaMA-7B-shaped set (61.9 M parameters)"
+    tiny = synth.Workload("llama7b_one", (synth.mat("wq", 4096, 4096), synth.vec("norm1", 4096)),
+                          synth.BF16, "normal_fixed", 1e-3, 0.0, (), 1, dict(synth.PAPER_HPARAMS))
+    return tiny, "one 4096x4096 matrix plus one 4096 vector of the LLaMA-7B-shaped set (16.8 M parameters)"
+
+
+def time_oracle(sample: synth.Workload, steps: int, warmup: int):
+    from oracle import came_oracle
+    params = synth.make_params(sample, 1)
+    orc = came_oracle.OracleOptimizer(params)
+    grads = [synth.widen(g) for g in synth.make_grads(sample, 1, 1)]
+    for _ in range(warmup):
+        orc.step(grads, **sample.hparams)
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        orc.step(grads, **sample.hparams)
+    dt = (time.perf_counter() - t0) / steps
+    return dt, came_oracle.threads()
+
+
+def cpu_baseline(budget_s: float, steps: int, warmup: int) -> dict:
+    sample, desc = _oracle_sample(budget_s, steps + warmup)
+    dt, threads = time_oracle(sample, steps, warmup)
+    return {"value": sample.numel / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
+            "sample": desc + f"; {steps} step(s), {dt:.2f} s per step; throughput per parameter is "
+                             "size-independent (tensors are independent)"}
+
+
+def run_reference(args):
+    rank, _, world = dist_env()
+    if rank != 0:
+        return
+    steps, warmup = args.steps, args.warmup
+    sample, desc = _oracle_sample(150.0, steps + warmup)
+    dt, threads = time_oracle(sample, steps, warmup)
+    value = sample.numel / dt
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
+            "steps": steps, "warmup": warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "sample": desc},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle",
+                             "sample": desc},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--workload", default="llama7b")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_gpu(args)
+
+
+if __name__ == "__main__":
+    main()

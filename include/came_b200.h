@@ -172,9 +172,11 @@ const char* came_status_string(came_status s);
 came_status came_query(const came_ctx* ctx, int32_t what, int64_t* out);
 
 /* Per-phase device timing.  When enabled, came_step records CUDA events on the
- * caller's stream between its kernels (no synchronisation).  came_get_phase_ms
- * synchronises on the last recorded event and writes up to `cap` durations in
- * milliseconds (HOST floats) in launch order; names via came_phase_name. */
+ * caller's stream between its kernels (no synchronisation); switching it on
+ * restarts the average.  came_get_phase_ms synchronises on the last recorded
+ * event and writes up to `cap` durations in milliseconds (HOST floats), each the
+ * mean over the profiled steps (the most recent 128), in launch order; names via
+ * came_phase_name. */
 came_status came_set_profiling(came_ctx* ctx, int32_t enabled);
 came_status came_get_phase_ms(came_ctx* ctx, float* out_ms, int32_t cap, int32_t* out_count);
 const char* came_phase_name(const came_ctx* ctx, int32_t phase);

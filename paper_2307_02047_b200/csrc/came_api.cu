@@ -20,6 +20,7 @@ using came::StepConsts;
 namespace {
 
 constexpr int kMaxPhases = 6;
+constexpr int kProfSlots = 128;        // profiled steps kept for averaging
 const char* const kPhaseNames[kMaxPhases] = {
     "vec_second_moment", "p1_reduce_g2", "p2_sum_u2", "p3_momentum_instability", "p4_apply",
     "vec_apply"};
@@ -95,10 +96,9 @@ struct came_ctx {
     long long numel = 0, matrix_numel = 0, state_bytes = 0, stream_bytes = 0, comp_bytes = 0;
     long long last_step = 0;
     bool profiling = false;
-    cudaEvent_t ev[kMaxPhases + 1] = {};
-    int phase_of_interval[kMaxPhases] = {};
+    std::vector<cudaEvent_t> prof_ev;          // [kProfSlots][kMaxPhases + 1], made on demand
+    long long prof_count = 0;                  // profiled steps since profiling was switched on
     int n_intervals = 0;
-    bool events_valid = false;
     std::string err;
 };
 
@@ -194,7 +194,7 @@ void free_ctx(came_ctx* ctx)
         if (ctx->pinned_table[k]) cudaFreeHost(ctx->pinned_table[k]);
         if (ctx->pinned_free[k]) cudaEventDestroy(ctx->pinned_free[k]);
     }
-    for (cudaEvent_t e : ctx->ev)
+    for (cudaEvent_t e : ctx->prof_ev)
         if (e) cudaEventDestroy(e);
     delete ctx;
 }
@@ -222,36 +222,37 @@ came_status upload_table(came_ctx* ctx, cudaStream_t stream)
 came_status launch_step(came_ctx* ctx, const came_hparams* hp, cudaStream_t stream)
 {
     const StepConsts hc = make_consts(*hp);
-    const bool prof = ctx->profiling;
+    const bool prof = ctx->profiling && !ctx->prof_ev.empty();
     int iv = 0;
-    auto mark = [&](int slot) { if (prof) cudaEventRecord(ctx->ev[slot], stream); };
+    cudaEvent_t* ev = prof ? &ctx->prof_ev[(ctx->prof_count % kProfSlots) * (kMaxPhases + 1)] : nullptr;
+    auto mark = [&](int slot) { if (prof) cudaEventRecord(ev[slot], stream); };
     mark(0);
     if (ctx->n_chunks > 0) {
         came::k_vec_second_moment<<<ctx->n_chunks, came::kThreads, 0, stream>>>(
             ctx->d_table, ctx->d_chunks, hc);
-        ctx->phase_of_interval[iv++] = 0; mark(iv);
+        mark(++iv);
     }
     if (ctx->n_tiles > 0) {
         came::k_p1_reduce_g2<<<ctx->n_tiles, came::kThreads, 0, stream>>>(
             ctx->d_table, ctx->d_tiles, ctx->n_tiles, 0, hc);
-        ctx->phase_of_interval[iv++] = 1; mark(iv);
+        mark(++iv);
         came::k_p2_sum_u2<<<ctx->n_tiles, came::kThreads, 0, stream>>>(
             ctx->d_table, ctx->d_tiles, ctx->n_tiles, 1, hc);
-        ctx->phase_of_interval[iv++] = 2; mark(iv);
+        mark(++iv);
         came::k_p3_momentum_instability<<<ctx->n_tiles, came::kThreads, 0, stream>>>(
             ctx->d_table, ctx->d_tiles, ctx->n_tiles, 0, hc);
-        ctx->phase_of_interval[iv++] = 3; mark(iv);
+        mark(++iv);
         came::k_p4_apply<<<ctx->n_tiles, came::kThreads, 0, stream>>>(
             ctx->d_table, ctx->d_tiles, ctx->n_tiles, 1, hc);
-        ctx->phase_of_interval[iv++] = 4; mark(iv);
+        mark(++iv);
     }
     if (ctx->n_chunks > 0) {
         came::k_vec_apply<<<ctx->n_chunks, came::kThreads, 0, stream>>>(
             ctx->d_table, ctx->d_chunks, hc);
-        ctx->phase_of_interval[iv++] = 5; mark(iv);
+        mark(++iv);
     }
     ctx->n_intervals = iv;
-    ctx->events_valid = prof;
+    if (prof) ++ctx->prof_count;
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(ctx, e, "kernel launch");
     ctx->last_step = hp->step;
@@ -412,7 +413,6 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
         CAME_TRY(cudaMallocHost(&ctx->pinned_table[k], ctx->table_bytes), "cudaMallocHost(table)");
         CAME_TRY(cudaEventCreateWithFlags(&ctx->pinned_free[k], cudaEventDisableTiming), "cudaEventCreate");
     }
-    for (cudaEvent_t& ev : ctx->ev) CAME_TRY(cudaEventCreate(&ev), "cudaEventCreate");
 
     for (int i = 0; i < n; ++i) {
         const came_tensor& x = t[i];
@@ -540,8 +540,16 @@ came_status came_query(const came_ctx* ctx, int32_t what, int64_t* out)
 came_status came_set_profiling(came_ctx* ctx, int32_t enabled)
 {
     if (!ctx) return CAME_ERR_NULL;
+    if (enabled && ctx->prof_ev.empty()) {
+        cudaSetDevice(ctx->device);
+        ctx->prof_ev.assign(static_cast<size_t>(kProfSlots) * (kMaxPhases + 1), nullptr);
+        for (cudaEvent_t& e : ctx->prof_ev) {
+            const cudaError_t err = cudaEventCreate(&e);
+            if (err != cudaSuccess) return cuda_fail(ctx, err, "cudaEventCreate");
+        }
+    }
     ctx->profiling = enabled != 0;
-    ctx->events_valid = false;
+    ctx->prof_count = 0;
     return CAME_OK;
 }
 
@@ -549,13 +557,22 @@ came_status came_get_phase_ms(came_ctx* ctx, float* out_ms, int32_t cap, int32_t
 {
     if (!ctx || !out_ms || !out_count) return CAME_ERR_NULL;
     *out_count = 0;
-    if (!ctx->events_valid) return fail(ctx, CAME_ERR_UNSUPPORTED, "no profiled step recorded");
-    cudaError_t e = cudaEventSynchronize(ctx->ev[ctx->n_intervals]);
+    if (ctx->prof_count == 0) return fail(ctx, CAME_ERR_UNSUPPORTED, "no profiled step recorded");
+    const int slots = static_cast<int>(std::min<long long>(ctx->prof_count, kProfSlots));
+    const int last = static_cast<int>((ctx->prof_count - 1) % kProfSlots);
+    cudaError_t e = cudaEventSynchronize(ctx->prof_ev[last * (kMaxPhases + 1) + ctx->n_intervals]);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaEventSynchronize");
     const int k = std::min<int>(cap, ctx->n_intervals);
     for (int i = 0; i < k; ++i) {
-        e = cudaEventElapsedTime(&out_ms[i], ctx->ev[i], ctx->ev[i + 1]);
-        if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaEventElapsedTime");
+        double sum = 0.0;
+        for (int sl = 0; sl < slots; ++sl) {
+            float ms = 0.f;
+            const cudaEvent_t* ev = &ctx->prof_ev[sl * (kMaxPhases + 1)];
+            e = cudaEventElapsedTime(&ms, ev[i], ev[i + 1]);
+            if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaEventElapsedTime");
+            sum += ms;
+        }
+        out_ms[i] = static_cast<float>(sum / slots);
     }
     *out_count = k;
     return CAME_OK;

@@ -24,7 +24,13 @@ def err_signed(x: np.ndarray, ref: np.ndarray) -> float:
 def err_positive(x: np.ndarray, ref: np.ndarray) -> float:
     """For the positive reductions r, c, R, C (and vector v, S): strict element-wise relative error."""
     ref = ref.astype(np.float64)
-    return float(np.max(np.abs(x.astype(np.float64) - ref) / ref))
+    x = x.astype(np.float64)
+    zero = ref == 0.0                      # untouched state (e.g. S of a no-confidence vector)
+    if np.any(x[zero] != 0.0):
+        return float("inf")
+    if zero.all():
+        return 0.0
+    return float(np.max(np.abs(x[~zero] - ref[~zero]) / ref[~zero]))
 
 
 def to_torch_grad(torch, g: np.ndarray, device):
@@ -39,6 +45,8 @@ def compare_state(opt, orc, indices=None) -> dict:
     idx = range(len(opt.params)) if indices is None else indices
     for k, i in enumerate(idx):
         j = i if indices is None else k
+        for a in (opt.params[i], opt.m[i]):
+            assert bool(a.isfinite().all()), "non-finite value in GPU state"
         worst["p"] = max(worst["p"], err_signed(opt.params[i].cpu().numpy(), orc.p[j]))
         worst["m"] = max(worst["m"], err_signed(opt.m[i].cpu().numpy(), orc.m[j]))
         worst["r"] = max(worst["r"], err_positive(opt.r[i].cpu().numpy(), orc.r[j]))
