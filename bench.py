@@ -184,7 +184,7 @@ def run_gpu(args):
     value = world * numel / (ms_per_step * 1e-3)
 
     # ---- end to end: host gradients in, updated parameters out, every step --------------
-    e2e = run_e2e(torch, binding, opt, w, hp, device, world, rank, args)
+    e2e = None if args.no_e2e else run_e2e(torch, binding, opt, w, hp, device, world, rank, args)
 
     peak, peak_kind = measured_peak()
     pb = phase_bytes(w)
@@ -380,6 +380,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

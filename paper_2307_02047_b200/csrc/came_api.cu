@@ -343,16 +343,16 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
         if (t[i].ndim == 2) matrix_numel += t[i].rows * t[i].cols;
     long long target = g_tile_elems_override;
     if (target <= 0) {
-        // aim for a few thousand tiles in all; between 4 Ki and 64 Ki elements per tile
+        // aim for a few thousand tiles in all; between 4 Ki and 256 Ki elements per tile
         target = 4096;
-        while (target < 65536 && target * 2 * 2400 <= matrix_numel) target *= 2;
+        while (target < 262144 && target * 2 * 2400 <= matrix_numel) target *= 2;
     }
     std::vector<Plan> plans(n);
     std::vector<Tile> tiles;
     std::vector<VChunk> chunks;
     size_t ws = 0;
     auto take = [&](size_t bytes) { const size_t off = ws; ws += (bytes + 255) / 256 * 256; return off; };
-    struct Off { size_t colpart, rowpart, blocksum, usq, cnt, scal; };
+    struct Off { size_t colpart, rowpart, blocksum, usq, cnt, scal, rowscale, colscale; };
     std::vector<Off> offs(n);
     for (int i = 0; i < n; ++i) {
         const came_tensor& x = t[i];
@@ -372,12 +372,15 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
             offs[i].colpart = take(sizeof(float) * static_cast<size_t>(p.n_rb) * x.cols);
             offs[i].rowpart = take(sizeof(float) * static_cast<size_t>(p.n_seg) * x.rows);
             offs[i].blocksum = take(sizeof(float) * p.n_rb);
+            offs[i].rowscale = take(sizeof(float) * static_cast<size_t>(x.rows));
+            offs[i].colscale = take(sizeof(float) * static_cast<size_t>(x.cols));
         } else {
             ctx->state_bytes += 4 * 3 * numel;
             ctx->stream_bytes += numel * (sg + 32);
             ctx->comp_bytes += numel * (sg + 32);
             for (int c = 0; c < p.n_parts; ++c) chunks.push_back(VChunk{i, c});
             offs[i].colpart = offs[i].rowpart = offs[i].blocksum = 0;
+            offs[i].rowscale = offs[i].colscale = 0;
         }
         offs[i].usq = take(sizeof(float) * p.n_parts);
         offs[i].cnt = take(sizeof(unsigned) * (p.n_rb + p.n_cb + 2));
@@ -425,6 +428,8 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
         d.ws_rowpart = reinterpret_cast<float*>(ctx->d_ws + offs[i].rowpart);
         d.ws_blocksum = reinterpret_cast<float*>(ctx->d_ws + offs[i].blocksum);
         d.ws_usq = reinterpret_cast<float*>(ctx->d_ws + offs[i].usq);
+        d.ws_rowscale = reinterpret_cast<float*>(ctx->d_ws + offs[i].rowscale);
+        d.ws_colscale = reinterpret_cast<float*>(ctx->d_ws + offs[i].colscale);
         d.cnt = reinterpret_cast<unsigned*>(ctx->d_ws + offs[i].cnt);
         d.scal = reinterpret_cast<float*>(ctx->d_ws + offs[i].scal);
         d.kind = p.kind; d.vec = p.vec;

@@ -9,7 +9,8 @@
 //   P3  g, m, r, c   -> m_t, row/column sums of (uhat - m_{t-1})^2 -> R_t, C_t, sqrt(1^T R_t)
 //   P4  m, theta, R, C -> theta_t
 // v_t and S_t (Eq. 2, rank one) are never formed: u = g * rsqrt(r_i) * sqrt(sum r) * rsqrt(c_j),
-// which also keeps r_i * c_j out of fp32 (it underflows for zero-gradient rows).
+// which also keeps r_i * c_j out of fp32 (it underflows for zero-gradient rows).  The
+// rsqrt of every finished row and column factor is stored once by the tile that finishes it.
 //
 // Reductions are deterministic: every tile writes its partial sums to a
 // workspace and the LAST tile to arrive (per row block, per column strip, per
@@ -20,6 +21,26 @@
 #include <stdint.h>
 
 namespace came {
+
+// Occupancy and unroll choices (resident blocks per SM, thread-rows in flight per thread).
+#ifndef CAME_P1_MINB
+#define CAME_P1_MINB 4
+#endif
+#ifndef CAME_P2_MINB
+#define CAME_P2_MINB 4
+#endif
+#ifndef CAME_P3_MINB
+#define CAME_P3_MINB 2
+#endif
+#ifndef CAME_P4_MINB
+#define CAME_P4_MINB 2
+#endif
+#ifndef CAME_P12_U
+#define CAME_P12_U 8
+#endif
+#ifndef CAME_P34_U
+#define CAME_P34_U 4
+#endif
 
 constexpr int kThreads = 256;
 constexpr int kVecChunk = 4096;       // vector elements per block in the vector kernels
@@ -39,6 +60,8 @@ struct TensorDev {
     float*       ws_rowpart;   // [n_seg][rows]  per-warp-segment row partial sums
     float*       ws_blocksum;  // [n_rb]         sum of the finished row factor over one row block
     float*       ws_usq;       // [n_parts]      per-tile partial sums of u^2
+    float*       ws_rowscale;  // [rows]  rsqrt of the row factor last finished (r_t, then R_t)
+    float*       ws_colscale;  // [cols]  rsqrt of the column factor last finished (c_t, then C_t)
     unsigned*    cnt;          // [n_rb] row-block arrivals, [n_cb] strip arrivals, [1] finished, [1] usq
     float*       scal;         // [0] sqrt(sum r)  [1] kappa  [2] sqrt(sum R)
     int          kind;
@@ -78,24 +101,6 @@ template <> struct Traits<kBF16x1> { static constexpr int VEC = 1; };
 
 __device__ __forceinline__ float bf16lo(uint32_t w) { return __uint_as_float(w << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
-
-// gradient load: read-only for the whole step
-template <int KIND>
-__device__ __forceinline__ void load_g(const void* base, long long idx, float (&x)[Traits<KIND>::VEC])
-{
-    if constexpr (KIND == kF32x4) {
-        const float4 v = __ldg(reinterpret_cast<const float4*>(static_cast<const float*>(base) + idx));
-        x[0] = v.x; x[1] = v.y; x[2] = v.z; x[3] = v.w;
-    } else if constexpr (KIND == kBF16x8) {
-        const uint4 v = __ldg(reinterpret_cast<const uint4*>(static_cast<const uint16_t*>(base) + idx));
-        x[0] = bf16lo(v.x); x[1] = bf16hi(v.x); x[2] = bf16lo(v.y); x[3] = bf16hi(v.y);
-        x[4] = bf16lo(v.z); x[5] = bf16hi(v.z); x[6] = bf16lo(v.w); x[7] = bf16hi(v.w);
-    } else if constexpr (KIND == kF32x1) {
-        x[0] = __ldg(static_cast<const float*>(base) + idx);
-    } else {
-        x[0] = __uint_as_float(static_cast<uint32_t>(__ldg(static_cast<const uint16_t*>(base) + idx)) << 16);
-    }
-}
 
 // fp32 state load/store: 1, 4 (128-bit) or 8 (256-bit, sm_100) floats per thread
 template <int VEC>
@@ -165,13 +170,41 @@ __device__ __forceinline__ T block_sum(T v, Shared& sm)
     return static_cast<T>(s);
 }
 
+// Sums U per-thread values across the 32 lanes of a warp with (U-1) + (5 - log2 U) shuffles.
+// On return every lane holds the full sum of v[k] for k = lane >> (5 - log2 U).
+template <int U>
+__device__ __forceinline__ float multi_row_warp_sum(float (&v)[U], int lane)
+{
+    int o = 16;
+#pragma unroll
+    for (int n = U; n > 1; n >>= 1, o >>= 1) {
+        const bool up = (lane & o) != 0;
+#pragma unroll
+        for (int i = 0; i < n / 2; ++i) {
+            const float keep = up ? v[i + n / 2] : v[i];
+            const float send = up ? v[i] : v[i + n / 2];
+            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, o);
+        }
+    }
+    float r = v[0];
+#pragma unroll
+    for (; o > 0; o >>= 1) r += __shfl_xor_sync(0xffffffffu, r, o);
+    return r;
+}
+
+template <int U> struct Log2;
+template <> struct Log2<1> { static constexpr int v = 0; };
+template <> struct Log2<2> { static constexpr int v = 1; };
+template <> struct Log2<4> { static constexpr int v = 2; };
+template <> struct Log2<8> { static constexpr int v = 3; };
+
 // ---------------------------------------------------------------------------
 // Last-arriver finalisation of one factored EMA (Algorithm 2: r_t, c_t from g^2
 // with beta2/eps1; R_t, C_t from U_t with beta3/eps2):
 //   row[i] = beta row[i] + (1-beta) (scale * sum_j X[i][j] + cols * eps)
 //   col[j] = beta col[j] + (1-beta) (scale * sum_i X[i][j] + rows * eps)
-// and, once every row block and strip of the tensor is finished,
-//   *sqrt_sum = sqrt(1_n^T row).
+// It also stores rsqrt(row[i]) and rsqrt(col[j]) for the phases that follow and,
+// once every row block and strip of the tensor is finished, *sqrt_sum = sqrt(1_n^T row).
 // Called by every tile of the tensor after it has written its partials.
 // ---------------------------------------------------------------------------
 __device__ __forceinline__ void finalize_factors(const TensorDev& d, int rb, int cb, float beta,
@@ -205,6 +238,7 @@ __device__ __forceinline__ void finalize_factors(const TensorDev& d, int rb, int
             for (int sg = 0; sg < d.n_seg; ++sg) s += __ldcg(d.ws_rowpart + sg * rows + row);
             const float nv = fmaf(beta, rowfac[row], omb * fmaf(scale, s, add));
             rowfac[row] = nv;
+            d.ws_rowscale[row] = __frsqrt_rn(nv);
             bs += nv;
         }
         bs = block_sum(bs, sm);
@@ -227,7 +261,9 @@ __device__ __forceinline__ void finalize_factors(const TensorDev& d, int rb, int
             }
             for (; k < d.n_rb; ++k) s0 += __ldcg(pc + k * cols);
             const float s = (s0 + s1) + (s2 + s3);
-            colfac[col] = fmaf(beta, colfac[col], omb * fmaf(scale, s, add));
+            const float nv = fmaf(beta, colfac[col], omb * fmaf(scale, s, add));
+            colfac[col] = nv;
+            d.ws_colscale[col] = __frsqrt_rn(nv);
         }
         if (tid == 0) d.cnt[d.n_rb + cb] = 0u;
     }
@@ -300,6 +336,47 @@ __device__ __forceinline__ Geo make_geo(const TensorDev& d, int rb, int cb)
     return q;
 }
 
+// raw gradient words of one thread-row: kept packed until they are used
+template <int KIND> struct Raw;
+template <> struct Raw<kF32x4>  { float4 v; };
+template <> struct Raw<kBF16x8> { uint4 v; };
+template <> struct Raw<kF32x1>  { float v; };
+template <> struct Raw<kBF16x1> { uint16_t v; };
+
+template <int KIND>
+__device__ __forceinline__ void load_raw(const char* p, Raw<KIND>& r)
+{
+    if constexpr (KIND == kF32x4) r.v = __ldg(reinterpret_cast<const float4*>(p));
+    else if constexpr (KIND == kBF16x8) r.v = __ldg(reinterpret_cast<const uint4*>(p));
+    else if constexpr (KIND == kF32x1) r.v = __ldg(reinterpret_cast<const float*>(p));
+    else r.v = __ldg(reinterpret_cast<const uint16_t*>(p));
+}
+
+template <int KIND>
+__device__ __forceinline__ void zero_raw(Raw<KIND>& r)
+{
+    if constexpr (KIND == kF32x4) r.v = make_float4(0.f, 0.f, 0.f, 0.f);
+    else if constexpr (KIND == kBF16x8) r.v = make_uint4(0u, 0u, 0u, 0u);
+    else if constexpr (KIND == kF32x1) r.v = 0.f;
+    else r.v = 0;
+}
+
+template <int KIND>
+__device__ __forceinline__ void unpack(const Raw<KIND>& r, float (&x)[Traits<KIND>::VEC])
+{
+    if constexpr (KIND == kF32x4) { x[0] = r.v.x; x[1] = r.v.y; x[2] = r.v.z; x[3] = r.v.w; }
+    else if constexpr (KIND == kBF16x8) {
+        x[0] = bf16lo(r.v.x); x[1] = bf16hi(r.v.x); x[2] = bf16lo(r.v.y); x[3] = bf16hi(r.v.y);
+        x[4] = bf16lo(r.v.z); x[5] = bf16hi(r.v.z); x[6] = bf16lo(r.v.w); x[7] = bf16hi(r.v.w);
+    } else if constexpr (KIND == kF32x1) x[0] = r.v;
+    else x[0] = __uint_as_float(static_cast<uint32_t>(r.v) << 16);
+}
+
+template <int KIND> __device__ __forceinline__ constexpr int grad_elem_bytes()
+{
+    return (KIND == kF32x4 || KIND == kF32x1) ? 4 : 2;
+}
+
 // write this tile's column partial sums (summed over the block's row groups in a fixed order)
 template <int VEC>
 __device__ __forceinline__ void write_col_partials(const TensorDev& d, const Geo& q, int rb,
@@ -325,6 +402,20 @@ __device__ __forceinline__ void write_col_partials(const TensorDev& d, const Geo
     if (q.colok) store_f<VEC>(d.ws_colpart + static_cast<long long>(rb) * d.cols + q.col, out);
 }
 
+// Row partial sums of U consecutive thread-rows (rows rbase + k*TY): reduced across the warp
+// in one batch; lane (k << (5 - log2 U)) stores row k's partial for this warp's column segment.
+template <int U>
+__device__ __forceinline__ void store_row_partials(float (&rs)[U], float* __restrict__ rowpart_seg,
+                                                   long long rbase, int TY, long long row1, int lane)
+{
+    constexpr int SH = 5 - Log2<U>::v;
+    const float tot = multi_row_warp_sum<U>(rs, lane);
+    if ((lane & ((1 << SH) - 1)) == 0) {
+        const long long row = rbase + static_cast<long long>(lane >> SH) * TY;
+        if (row < row1) rowpart_seg[row] = tot;
+    }
+}
+
 // ---------------------------------------------------------------------------
 // P1 (Algorithm 2: r_t, c_t): row and column sums of g^2
 // ---------------------------------------------------------------------------
@@ -333,37 +424,46 @@ __device__ __forceinline__ void p1_tile(const TensorDev& d, int rb, int cb, cons
                                         Shared& sm)
 {
     constexpr int VEC = Traits<KIND>::VEC;
-    constexpr int U = 8;
+    constexpr int U = CAME_P12_U;
     const Geo q = make_geo<VEC>(d, rb, cb);
-    const long long cols = d.cols;
     const int lane = threadIdx.x & 31;
+    const long long stride = static_cast<long long>(q.TY) * d.cols * grad_elem_bytes<KIND>();
+    const char* gp = static_cast<const char*>(d.g) +
+                     ((q.row0 + q.ty) * d.cols + q.col) * grad_elem_bytes<KIND>();
+    float* const rowpart_seg = d.ws_rowpart + q.seg * d.rows;
     float cacc[VEC];
 #pragma unroll
     for (int v = 0; v < VEC; ++v) cacc[v] = 0.f;
 
     for (long long rbase = q.row0 + q.ty; rbase < q.row1; rbase += static_cast<long long>(q.TY) * U) {
-        float x[U][VEC];
+        Raw<KIND> raw[U];
+        const bool full = rbase + static_cast<long long>(U - 1) * q.TY < q.row1;
+        if (full && q.colok) {
 #pragma unroll
-        for (int k = 0; k < U; ++k) {
-            const long long row = rbase + static_cast<long long>(k) * q.TY;
-            if (row < q.row1 && q.colok) load_g<KIND>(d.g, row * cols + q.col, x[k]);
-            else {
+            for (int k = 0; k < U; ++k) load_raw<KIND>(gp + k * stride, raw[k]);
+        } else {
 #pragma unroll
-                for (int v = 0; v < VEC; ++v) x[k][v] = 0.f;
+            for (int k = 0; k < U; ++k) {
+                if (q.colok && rbase + static_cast<long long>(k) * q.TY < q.row1)
+                    load_raw<KIND>(gp + k * stride, raw[k]);
+                else zero_raw<KIND>(raw[k]);
             }
         }
+        gp += U * stride;
+        float rs[U];
 #pragma unroll
         for (int k = 0; k < U; ++k) {
-            const long long row = rbase + static_cast<long long>(k) * q.TY;
-            float rs = 0.f;
+            float x[VEC];
+            unpack<KIND>(raw[k], x);
+            float s = 0.f;
 #pragma unroll
             for (int v = 0; v < VEC; ++v) {
-                cacc[v] = fmaf(x[k][v], x[k][v], cacc[v]);
-                rs = fmaf(x[k][v], x[k][v], rs);
+                cacc[v] = fmaf(x[v], x[v], cacc[v]);
+                s = fmaf(x[v], x[v], s);
             }
-            rs = warp_sum(rs);
-            if (lane == 0 && row < q.row1) d.ws_rowpart[q.seg * d.rows + row] = rs;
+            rs[k] = s;
         }
+        store_row_partials<U>(rs, rowpart_seg, rbase, q.TY, q.row1, lane);
     }
     write_col_partials<VEC>(d, q, rb, cacc, sm);
     finalize_factors(d, rb, cb, hc.beta2, hc.omb2, hc.eps1, 1.0f, d.r, d.c, d.scal + 0, sm);
@@ -377,35 +477,43 @@ __device__ __forceinline__ void p2_tile(const TensorDev& d, int rb, int cb, cons
                                         Shared& sm)
 {
     constexpr int VEC = Traits<KIND>::VEC;
-    constexpr int U = 8;
+    constexpr int U = CAME_P12_U;
     const Geo q = make_geo<VEC>(d, rb, cb);
-    const long long cols = d.cols;
+    const long long stride = static_cast<long long>(q.TY) * d.cols * grad_elem_bytes<KIND>();
+    const char* gp = static_cast<const char*>(d.g) +
+                     ((q.row0 + q.ty) * d.cols + q.col) * grad_elem_bytes<KIND>();
+    const float* ap = d.ws_rowscale + q.row0 + q.ty;
     const float ssr = d.scal[0];
     float b[VEC];
 #pragma unroll
-    for (int v = 0; v < VEC; ++v) b[v] = q.colok ? __frsqrt_rn(d.c[q.col + v]) : 0.f;
+    for (int v = 0; v < VEC; ++v) b[v] = q.colok ? d.ws_colscale[q.col + v] : 0.f;
     float acc = 0.f;
 
     for (long long rbase = q.row0 + q.ty; rbase < q.row1; rbase += static_cast<long long>(q.TY) * U) {
-        float x[U][VEC];
+        Raw<KIND> raw[U];
         float a[U];
+        const bool full = rbase + static_cast<long long>(U - 1) * q.TY < q.row1;
+        if (full && q.colok) {
 #pragma unroll
-        for (int k = 0; k < U; ++k) {
-            const long long row = rbase + static_cast<long long>(k) * q.TY;
-            const bool ok = row < q.row1;
-            a[k] = ok ? d.r[row] : 1.f;
-            if (ok && q.colok) load_g<KIND>(d.g, row * cols + q.col, x[k]);
-            else {
+            for (int k = 0; k < U; ++k) { load_raw<KIND>(gp + k * stride, raw[k]); a[k] = ap[k * q.TY]; }
+        } else {
 #pragma unroll
-                for (int v = 0; v < VEC; ++v) x[k][v] = 0.f;
+            for (int k = 0; k < U; ++k) {
+                if (q.colok && rbase + static_cast<long long>(k) * q.TY < q.row1) {
+                    load_raw<KIND>(gp + k * stride, raw[k]); a[k] = ap[k * q.TY];
+                } else { zero_raw<KIND>(raw[k]); a[k] = 0.f; }
             }
         }
+        gp += U * stride;
+        ap += U * q.TY;
 #pragma unroll
         for (int k = 0; k < U; ++k) {
-            const float ai = __frsqrt_rn(a[k]) * ssr;
+            float x[VEC];
+            unpack<KIND>(raw[k], x);
+            const float ai = a[k] * ssr;
 #pragma unroll
             for (int v = 0; v < VEC; ++v) {
-                const float u = (x[k][v] * b[v]) * ai;
+                const float u = (x[v] * b[v]) * ai;
                 acc = fmaf(u, u, acc);
             }
         }
@@ -424,51 +532,74 @@ __device__ __forceinline__ void p3_tile(const TensorDev& d, int rb, int cb, cons
                                         Shared& sm)
 {
     constexpr int VEC = Traits<KIND>::VEC;
-    constexpr int U = 4;
+    constexpr int U = CAME_P34_U;
     const Geo q = make_geo<VEC>(d, rb, cb);
-    const long long cols = d.cols;
     const int lane = threadIdx.x & 31;
+    const long long first = (q.row0 + q.ty) * d.cols + q.col;
+    const long long gstride = static_cast<long long>(q.TY) * d.cols * grad_elem_bytes<KIND>();
+    const long long mstride = static_cast<long long>(q.TY) * d.cols;
+    const char* gp = static_cast<const char*>(d.g) + first * grad_elem_bytes<KIND>();
+    float* mp = d.m + first;
+    const float* ap = d.ws_rowscale + q.row0 + q.ty;
+    float* const rowpart_seg = d.ws_rowpart + q.seg * d.rows;
     const float ssr_k = d.scal[0] * d.scal[1];          // sqrt(sum r) * kappa
+    const float omb1 = hc.omb1;
     float b[VEC], cacc[VEC];
 #pragma unroll
     for (int v = 0; v < VEC; ++v) {
-        b[v] = q.colok ? __frsqrt_rn(d.c[q.col + v]) : 0.f;
+        b[v] = q.colok ? d.ws_colscale[q.col + v] : 0.f;
         cacc[v] = 0.f;
     }
 
     for (long long rbase = q.row0 + q.ty; rbase < q.row1; rbase += static_cast<long long>(q.TY) * U) {
-        float x[U][VEC], mo[U][VEC], a[U];
+        Raw<KIND> raw[U];
+        float mo[U][VEC], a[U];
+        const bool full = rbase + static_cast<long long>(U - 1) * q.TY < q.row1;
+        if (full && q.colok) {
 #pragma unroll
-        for (int k = 0; k < U; ++k) {
-            const long long row = rbase + static_cast<long long>(k) * q.TY;
-            const bool ok = row < q.row1;
-            a[k] = ok ? d.r[row] : 1.f;
-            if (ok && q.colok) {
-                load_g<KIND>(d.g, row * cols + q.col, x[k]);
-                load_f<VEC>(d.m + row * cols + q.col, mo[k]);
-            } else {
+            for (int k = 0; k < U; ++k) {
+                load_raw<KIND>(gp + k * gstride, raw[k]);
+                load_f<VEC>(mp + k * mstride, mo[k]);
+                a[k] = ap[k * q.TY];
+            }
+        } else {
 #pragma unroll
-                for (int v = 0; v < VEC; ++v) { x[k][v] = 0.f; mo[k][v] = 0.f; }
+            for (int k = 0; k < U; ++k) {
+                if (q.colok && rbase + static_cast<long long>(k) * q.TY < q.row1) {
+                    load_raw<KIND>(gp + k * gstride, raw[k]);
+                    load_f<VEC>(mp + k * mstride, mo[k]);
+                    a[k] = ap[k * q.TY];
+                } else {
+                    zero_raw<KIND>(raw[k]);
+                    a[k] = 0.f;
+#pragma unroll
+                    for (int v = 0; v < VEC; ++v) mo[k][v] = 0.f;
+                }
             }
         }
+        float rs[U];
 #pragma unroll
         for (int k = 0; k < U; ++k) {
-            const long long row = rbase + static_cast<long long>(k) * q.TY;
-            const bool ok = row < q.row1;
-            const float ai = __frsqrt_rn(a[k]) * ssr_k;
-            float rs = 0.f;
+            float x[VEC];
+            unpack<KIND>(raw[k], x);
+            const float ai = a[k] * ssr_k;
+            float s = 0.f;
 #pragma unroll
             for (int v = 0; v < VEC; ++v) {
-                const float uh = (x[k][v] * b[v]) * ai;
+                const float uh = (x[v] * b[v]) * ai;
                 const float e = uh - mo[k][v];
-                mo[k][v] = fmaf(hc.omb1, e, mo[k][v]);
+                mo[k][v] = fmaf(omb1, e, mo[k][v]);
                 cacc[v] = fmaf(e, e, cacc[v]);
-                rs = fmaf(e, e, rs);
+                s = fmaf(e, e, s);
             }
-            if (ok && q.colok) store_f<VEC>(d.m + row * cols + q.col, mo[k]);
-            rs = warp_sum(rs);
-            if (lane == 0 && ok) d.ws_rowpart[q.seg * d.rows + row] = rs;
+            rs[k] = s;
+            if (q.colok && (full || rbase + static_cast<long long>(k) * q.TY < q.row1))
+                store_f<VEC>(mp + k * mstride, mo[k]);
         }
+        gp += U * gstride;
+        mp += U * mstride;
+        ap += U * q.TY;
+        store_row_partials<U>(rs, rowpart_seg, rbase, q.TY, q.row1, lane);
     }
     write_col_partials<VEC>(d, q, rb, cacc, sm);
     finalize_factors(d, rb, cb, hc.beta3, hc.omb3, hc.eps2, hc.b1sq, d.R, d.C, d.scal + 2, sm);
@@ -482,41 +613,47 @@ template <int KIND>
 __device__ __forceinline__ void p4_tile(const TensorDev& d, int rb, int cb, const StepConsts& hc)
 {
     constexpr int VEC = Traits<KIND>::VEC;
-    constexpr int U = 4;
+    constexpr int U = CAME_P34_U;
     const Geo q = make_geo<VEC>(d, rb, cb);
     if (!q.colok) return;
-    const long long cols = d.cols;
+    const long long first = (q.row0 + q.ty) * d.cols + q.col;
+    const long long stride = static_cast<long long>(q.TY) * d.cols;
+    const float* mp = d.m + first;
+    float* pp = d.p + first;
+    const float* ap = d.ws_rowscale + q.row0 + q.ty;
     const float ssR = d.scal[2];
     const float wd = (d.flags & kFlagNoWd) ? 0.f : hc.wd;
+    const float nlr = -hc.lr;
     float B[VEC];
 #pragma unroll
-    for (int v = 0; v < VEC; ++v) B[v] = __frsqrt_rn(d.C[q.col + v]);
+    for (int v = 0; v < VEC; ++v) B[v] = d.ws_colscale[q.col + v];
 
     for (long long rbase = q.row0 + q.ty; rbase < q.row1; rbase += static_cast<long long>(q.TY) * U) {
         float mo[U][VEC], th[U][VEC], a[U];
+        const bool full = rbase + static_cast<long long>(U - 1) * q.TY < q.row1;
 #pragma unroll
         for (int k = 0; k < U; ++k) {
-            const long long row = rbase + static_cast<long long>(k) * q.TY;
-            const bool ok = row < q.row1;
-            a[k] = ok ? d.R[row] : 1.f;
-            if (ok) {
-                load_f<VEC>(d.m + row * cols + q.col, mo[k]);
-                load_f<VEC>(d.p + row * cols + q.col, th[k]);
+            if (full || rbase + static_cast<long long>(k) * q.TY < q.row1) {
+                load_f<VEC>(mp + k * stride, mo[k]);
+                load_f<VEC>(pp + k * stride, th[k]);
+                a[k] = ap[k * q.TY];
             }
         }
 #pragma unroll
         for (int k = 0; k < U; ++k) {
-            const long long row = rbase + static_cast<long long>(k) * q.TY;
-            if (row < q.row1) {
-                const float Ai = __frsqrt_rn(a[k]) * ssR;
+            if (full || rbase + static_cast<long long>(k) * q.TY < q.row1) {
+                const float Ai = a[k] * ssR;
 #pragma unroll
                 for (int v = 0; v < VEC; ++v) {
                     const float upd = fmaf(wd, th[k][v], (mo[k][v] * B[v]) * Ai);
-                    th[k][v] = fmaf(-hc.lr, upd, th[k][v]);
+                    th[k][v] = fmaf(nlr, upd, th[k][v]);
                 }
-                store_f<VEC>(d.p + row * cols + q.col, th[k]);
+                store_f<VEC>(pp + k * stride, th[k]);
             }
         }
+        mp += U * stride;
+        pp += U * stride;
+        ap += U * q.TY;
     }
 }
 
@@ -537,42 +674,42 @@ __device__ __forceinline__ Tile fetch_tile(const Tile* tiles, int ntiles, int re
     return tiles[reverse ? (ntiles - 1 - b) : b];
 }
 
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, CAME_P1_MINB)
 k_p1_reduce_g2(const TensorDev* __restrict__ T, const Tile* __restrict__ tiles, int ntiles,
                int reverse, StepConsts hc)
 {
     __shared__ Shared sm;
     const Tile t = fetch_tile(tiles, ntiles, reverse);
-    const TensorDev& d = T[t.tensor];
+    const TensorDev d = T[t.tensor];       // by value: descriptor fields live in registers
     CAME_DISPATCH(p1_tile, d, t.rb, t.cb, hc, sm)
 }
 
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, CAME_P2_MINB)
 k_p2_sum_u2(const TensorDev* __restrict__ T, const Tile* __restrict__ tiles, int ntiles,
             int reverse, StepConsts hc)
 {
     __shared__ Shared sm;
     const Tile t = fetch_tile(tiles, ntiles, reverse);
-    const TensorDev& d = T[t.tensor];
+    const TensorDev d = T[t.tensor];
     CAME_DISPATCH(p2_tile, d, t.rb, t.cb, hc, sm)
 }
 
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, CAME_P3_MINB)
 k_p3_momentum_instability(const TensorDev* __restrict__ T, const Tile* __restrict__ tiles,
                           int ntiles, int reverse, StepConsts hc)
 {
     __shared__ Shared sm;
     const Tile t = fetch_tile(tiles, ntiles, reverse);
-    const TensorDev& d = T[t.tensor];
+    const TensorDev d = T[t.tensor];
     CAME_DISPATCH(p3_tile, d, t.rb, t.cb, hc, sm)
 }
 
-__global__ void __launch_bounds__(kThreads, 2)
+__global__ void __launch_bounds__(kThreads, CAME_P4_MINB)
 k_p4_apply(const TensorDev* __restrict__ T, const Tile* __restrict__ tiles, int ntiles,
            int reverse, StepConsts hc)
 {
     const Tile t = fetch_tile(tiles, ntiles, reverse);
-    const TensorDev& d = T[t.tensor];
+    const TensorDev d = T[t.tensor];
     CAME_DISPATCH(p4_tile, d, t.rb, t.cb, hc)
 }
 
