@@ -191,6 +191,37 @@ came_status came_plan_tensor(int64_t rows, int64_t cols, int32_t ndim, int32_t g
                              int32_t* out_threads_x, int32_t* out_tile_rows, int32_t* out_n_rb,
                              int32_t* out_n_cb);
 
+/* Allocation-free factor update (the paper has no counterpart: this exists for callers of
+ * this library that are not allowed to allocate device memory).
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- inside a memory pool or
+ * framework allocator that owns the whole device heap, in a latency-critical loop where an
+ * allocation's implicit synchronisation is unacceptable, or under a fixed memory budget
+ * audited at start-up.  Such a caller cannot use came_create, which allocates the context's
+ * tables and reduction workspace.
+ *
+ * What it does: the first two lines of Algorithm 2 for ONE matrix,
+ *   r = beta2 r + (1-beta2)(g^2 + eps1 1 1^T) 1_m,   c = beta2 c + (1-beta2) 1_n^T (g^2 + eps1 1 1^T),
+ * with the same tile kernel as came_step's first phase.  `grad` (DEVICE, grad_dtype
+ * [rows*cols], row-major, 16-byte aligned, read only), `r` (DEVICE fp32 [rows], in/out),
+ * `c` (DEVICE fp32 [cols], in/out); `out_sqrt_sum_r` (DEVICE fp32 [1], may be NULL)
+ * receives sqrt(1_n^T r).  The partial sums live in a fixed array of
+ * CAME_STATIC_SCRATCH_BYTES inside the library image (every GPU that loads the library
+ * holds that much until the process exits).  A matrix whose partial sums do not fit is
+ * rejected with CAME_ERR_UNSUPPORTED and a message naming the bytes needed; nothing is
+ * launched.  Calls no cudaMalloc, cudaFree or other allocating routine.
+ *
+ * The first call on each device looks up the device address of the scratch array (a
+ * cudaGetSymbolAddress with `device` current); make that first call outside any stream
+ * capture.  Every call uses the same scratch array and clears the part that must start at
+ * zero, so two calls whose GPU work overlaps (different streams, or different host threads)
+ * race: serialise them on one stream.  Asynchronous on `cuda_stream`. */
+#define CAME_STATIC_SCRATCH_BYTES (8u << 20)
+came_status came_factor_update_static(const void* grad, int32_t grad_dtype, int64_t rows,
+                                      int64_t cols, float* r, float* c, double beta2,
+                                      double eps1, float* out_sqrt_sum_r, int32_t device,
+                                      void* cuda_stream);
+
 /* Process-wide tuning knob, read by later came_create calls.  CAME_TUNE_TILE_ELEMS:
  * elements per matrix tile (0 restores the default, which scales with the size
  * of the parameter set).  Changes scheduling only, never results beyond the

@@ -27,7 +27,7 @@ CAME_TUNE_TILE_ELEMS = 0
 
 EXPORTED = ["came_create", "came_step", "came_step_host", "came_destroy", "came_last_error",
             "came_status_string", "came_query", "came_set_profiling", "came_get_phase_ms",
-            "came_phase_name", "came_plan_tensor", "came_tune"]
+            "came_phase_name", "came_plan_tensor", "came_tune", "came_factor_update_static"]
 
 
 class CameError(RuntimeError):
@@ -87,6 +87,9 @@ def load():
     L.came_plan_tensor.restype = i32
     L.came_tune.argtypes = [i32, i64]
     L.came_tune.restype = i32
+    L.came_factor_update_static.argtypes = [vp, i32, i64, i64, vp, vp, ctypes.c_double,
+                                            ctypes.c_double, vp, i32, vp]
+    L.came_factor_update_static.restype = i32
     _lib = L
     return L
 
@@ -169,6 +172,24 @@ def came_plan_tensor(rows: int, cols: int, ndim: int, grad_dtype: int, aligned32
 
 def came_tune(key: int, value: int) -> None:
     _check(load().came_tune(key, value))
+
+
+CAME_STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def came_factor_update_static(grad: int, grad_dtype: int, rows: int, cols: int, r: int, c: int,
+                              beta2: float, eps1: float, out_sqrt_sum_r: Optional[int] = None,
+                              device: int = 0, stream: int = 0) -> None:
+    """r, c <- the first two lines of Algorithm 2 for one matrix, without any allocation.
+
+    For callers that may not allocate device memory (an allocator that owns the device
+    heap, a no-synchronisation loop, an audited memory budget): the partial sums use a
+    fixed array inside the library instead of a context's workspace.  All pointer
+    arguments are device addresses (ints).  Calls share that array: keep them on one stream.
+    """
+    _check(load().came_factor_update_static(grad, grad_dtype, rows, cols, r, c, float(beta2),
+                                            float(eps1), out_sqrt_sum_r, device,
+                                            ctypes.c_void_p(stream)))
 
 
 def make_hparams(step: int, **kw) -> came_hparams:

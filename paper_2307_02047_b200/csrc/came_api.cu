@@ -599,3 +599,125 @@ const char* came_phase_name(const came_ctx* ctx, int32_t phase)
 }
 
 }  // extern "C"
+
+// =============================================================================================
+// Allocation-free factor update (came_factor_update_static).  Everything it needs on the
+// device beyond the caller's buffers lives in g_static_scratch below.
+// =============================================================================================
+namespace {
+
+// Partial sums, finished-factor scales, arrival counters and scalars of ONE matrix.
+// Device memory owned by the library image; see the header for the sharing rules.
+static __device__ __align__(256) unsigned char g_static_scratch[CAME_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_addr[kMaxDevices] = {};   // device address of g_static_scratch, per device
+
+// One block per tile of the single matrix described by `d` (passed by value): the tile
+// indices come from the block index, so no device-resident table or tile list is needed.
+__global__ void __launch_bounds__(came::kThreads, CAME_P1_MINB)
+k_p1_reduce_g2_single(const TensorDev d, StepConsts hc)
+{
+    __shared__ came::Shared sm;
+    const int rb = static_cast<int>(blockIdx.x) / d.n_cb;
+    const int cb = static_cast<int>(blockIdx.x) % d.n_cb;
+    using namespace came;
+    CAME_DISPATCH(p1_tile, d, rb, cb, hc, sm)
+}
+
+}  // namespace
+
+extern "C" came_status came_factor_update_static(const void* grad, int32_t grad_dtype, int64_t rows,
+                                                 int64_t cols, float* r, float* c, double beta2,
+                                                 double eps1, float* out_sqrt_sum_r, int32_t device,
+                                                 void* cuda_stream)
+{
+    if (!grad || !r || !c) return fail(nullptr, CAME_ERR_NULL, "grad, r and c are required");
+    if (rows < 1 || cols < 1 || rows > (1ll << 40) / cols)
+        return fail(nullptr, CAME_ERR_SHAPE, "rows and cols must be >= 1 and rows*cols <= 2^40");
+    if (grad_dtype != CAME_F32 && grad_dtype != CAME_BF16)
+        return fail(nullptr, CAME_ERR_DTYPE, "unknown grad_dtype");
+    if (!aligned(grad, 16) || !aligned(r, 16) || !aligned(c, 16))
+        return fail(nullptr, CAME_ERR_ALIGN, "pointer not 16-byte aligned");
+    if (!std::isfinite(beta2) || beta2 < 0.0 || beta2 >= 1.0 || !std::isfinite(eps1) || eps1 < 0.0)
+        return fail(nullptr, CAME_ERR_HPARAM, "beta2 must lie in [0,1) and eps1 must be >= 0");
+    if (device < 0 || device >= kMaxDevices)
+        return fail(nullptr, CAME_ERR_DEVICE, "device ordinal out of range");
+
+    // Lay the scratch out; grow the tile until the partial sums fit (fewer, taller tiles).
+    Plan p;
+    size_t need = 0;
+    struct { size_t colpart, rowpart, blocksum, rowscale, colscale, cnt, scal; } off{};
+    for (long long target = 32768; ; target *= 2) {
+        p = plan_tensor(rows, cols, 2, grad_dtype, true, target);
+        size_t ws = 0;
+        auto take = [&](size_t bytes) { const size_t o = ws; ws += (bytes + 255) / 256 * 256; return o; };
+        off.cnt = take(sizeof(unsigned) * (static_cast<size_t>(p.n_rb) + p.n_cb + 2));
+        off.scal = take(sizeof(float) * 4);
+        off.blocksum = take(sizeof(float) * p.n_rb);
+        off.colpart = take(sizeof(float) * static_cast<size_t>(p.n_rb) * cols);
+        off.rowpart = take(sizeof(float) * static_cast<size_t>(p.n_seg) * rows);
+        off.rowscale = take(sizeof(float) * static_cast<size_t>(rows));
+        off.colscale = take(sizeof(float) * static_cast<size_t>(cols));
+        need = ws;
+        if (need <= CAME_STATIC_SCRATCH_BYTES || p.n_rb == 1 || target >= (1ll << 40)) break;
+    }
+    if (need > CAME_STATIC_SCRATCH_BYTES) {
+        char buf[200];
+        std::snprintf(buf, sizeof buf,
+                      "matrix %lld x %lld needs %zu bytes of partial sums; the built-in scratch holds %u",
+                      static_cast<long long>(rows), static_cast<long long>(cols), need,
+                      static_cast<unsigned>(CAME_STATIC_SCRATCH_BYTES));
+        return fail(nullptr, CAME_ERR_UNSUPPORTED, buf);
+    }
+    if (static_cast<long long>(p.n_rb) * p.n_cb > (1ll << 30))
+        return fail(nullptr, CAME_ERR_SHAPE, "too many tiles");
+
+    cudaError_t e = cudaSetDevice(device);
+    if (e != cudaSuccess) { cudaGetLastError(); return fail(nullptr, CAME_ERR_DEVICE, "cudaSetDevice failed"); }
+    if (!g_static_scratch_addr[device]) {
+        // The array's name is only a host-side handle; kernels need its device address.
+        void* ptr = nullptr;
+        e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+        if (e != cudaSuccess) return cuda_fail(nullptr, e, "cudaGetSymbolAddress(scratch)");
+        g_static_scratch_addr[device] = ptr;
+    }
+    char* base = static_cast<char*>(g_static_scratch_addr[device]);
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+    // The arrival counters and scalars must start at zero whatever the last call left behind.
+    e = cudaMemsetAsync(base, 0, off.blocksum, stream);
+    if (e != cudaSuccess) return cuda_fail(nullptr, e, "cudaMemsetAsync(scratch counters)");
+
+    TensorDev d;
+    std::memset(&d, 0, sizeof d);
+    d.g = grad; d.r = r; d.c = c;
+    d.rows = rows; d.cols = cols;
+    d.cnt = reinterpret_cast<unsigned*>(base + off.cnt);
+    d.scal = reinterpret_cast<float*>(base + off.scal);
+    d.ws_blocksum = reinterpret_cast<float*>(base + off.blocksum);
+    d.ws_colpart = reinterpret_cast<float*>(base + off.colpart);
+    d.ws_rowpart = reinterpret_cast<float*>(base + off.rowpart);
+    d.ws_rowscale = reinterpret_cast<float*>(base + off.rowscale);
+    d.ws_colscale = reinterpret_cast<float*>(base + off.colscale);
+    d.ws_usq = d.scal;          // unused by this phase
+    d.kind = p.kind; d.vec = p.vec;
+    int lg = 0; while ((1 << lg) < p.tx) ++lg;
+    d.tx_log2 = lg; d.tr = p.tr; d.n_rb = p.n_rb; d.n_cb = p.n_cb; d.n_seg = p.n_seg;
+    d.n_parts = p.n_parts; d.ndim = 2; d.flags = 0;
+
+    StepConsts hc;
+    std::memset(&hc, 0, sizeof hc);
+    hc.beta2 = static_cast<float>(beta2);
+    hc.omb2 = static_cast<float>(1.0 - beta2);
+    hc.eps1 = static_cast<float>(eps1);
+    hc.clip_d = 1.0;
+    k_p1_reduce_g2_single<<<p.n_rb * p.n_cb, came::kThreads, 0, stream>>>(d, hc);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(nullptr, e, "kernel launch");
+    if (out_sqrt_sum_r) {
+        e = cudaMemcpyAsync(out_sqrt_sum_r, d.scal, sizeof(float), cudaMemcpyDeviceToDevice, stream);
+        if (e != cudaSuccess) return cuda_fail(nullptr, e, "cudaMemcpyAsync(sqrt sum r)");
+    }
+    return CAME_OK;
+}
