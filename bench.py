@@ -230,7 +230,13 @@ def run_gpu(args):
 
 # ncu-measured DRAM bytes per launch of the dominant kernel (read + write), keyed by
 # (workload, kernel).  None until a capture of the current kernel exists.
-TRAFFIC_BYTES = {}
+TRAFFIC_BYTES = {
+    # one-layer capture (profiles/ncu_phase_kernels_llama7b_layer.md) scaled by matrix elements
+    ("llama7b", "p4_apply"): 79.35e9,
+    ("llama7b", "p3_momentum_instability"): 67.44e9,
+    ("llama7b_layer", "p4_apply"): 2.3832e9,
+    ("llama7b_layer", "p3_momentum_instability"): 2.0254e9,
+}
 
 
 def host_mem_available() -> int:
