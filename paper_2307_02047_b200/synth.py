@@ -234,9 +234,15 @@ def make_grad(w: Workload, seed: int, i: int, step: int) -> np.ndarray:
     return g.astype(np.float32, copy=False)
 
 
-def make_grads(w: Workload, seed: int, step: int, indices: Sequence[int] | None = None
-               ) -> List[np.ndarray]:
-    idx = range(len(w.tensors)) if indices is None else indices
+def make_grads(w: Workload, seed: int, step: int, indices: Sequence[int] | None = None,
+               workers: int = 0) -> List[np.ndarray]:
+    """All (or the listed) gradients of one step.  Draws are keyed per tensor, so generating
+    them on ``workers`` threads gives the same bits as generating them one by one."""
+    idx = list(range(len(w.tensors)) if indices is None else indices)
+    if workers > 1 and len(idx) > 1:
+        from concurrent.futures import ThreadPoolExecutor
+        with ThreadPoolExecutor(max_workers=workers) as ex:
+            return list(ex.map(lambda i: make_grad(w, seed, i, step), idx))
     return [make_grad(w, seed, i, step) for i in idx]
 
 

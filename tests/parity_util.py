@@ -58,27 +58,35 @@ def compare_state(opt, orc, indices=None) -> dict:
 
 
 def run_paired(torch, binding, oracle, w: synth.Workload, seed: int, steps: int, check_at,
-               flags=None, hparams=None, device="cuda:0"):
-    """Step the CUDA path and the oracle side by side; returns {step: worst-error dict}."""
+               flags=None, hparams=None, device="cuda:0", oracle_idx=None, workers: int = 0):
+    """Step the CUDA path and the oracle side by side; returns {step: worst-error dict}.
+
+    ``oracle_idx``: run the oracle on these tensors only (tensors are independent, so each is
+    an exact element-by-element check of the full-size GPU run); None = all tensors.
+    """
     hp = dict(w.hparams if hparams is None else hparams)
     params = synth.make_params(w, seed)
-    dev_p = [torch.from_numpy(p.copy()).to(device) for p in params]
-    g0 = synth.make_grads(w, seed, 1)
+    dev_p = [torch.from_numpy(p).to(device) for p in params]
+    g0 = synth.make_grads(w, seed, 1, workers=workers)
     dev_g = [to_torch_grad(torch, g, device) for g in g0]
     opt = binding.CameOptimizer(dev_p, dev_g, flags=flags)
-    no_wd = [bool(f & binding.CAME_T_NO_WEIGHT_DECAY) for f in flags] if flags else ()
-    no_conf = [bool(f & binding.CAME_T_VEC_NO_CONFIDENCE) for f in flags] if flags else ()
-    orc = oracle.OracleOptimizer(params, no_weight_decay=no_wd, vec_no_confidence=no_conf)
+    sel = list(range(len(params))) if oracle_idx is None else list(oracle_idx)
+    no_wd = [bool(flags[i] & binding.CAME_T_NO_WEIGHT_DECAY) for i in sel] if flags else ()
+    no_conf = [bool(flags[i] & binding.CAME_T_VEC_NO_CONFIDENCE) for i in sel] if flags else ()
+    orc = oracle.OracleOptimizer([params[i] for i in sel], no_weight_decay=no_wd,
+                                 vec_no_confidence=no_conf)
+    del params
     out = {}
     for step in range(1, steps + 1):
-        grads = g0 if step == 1 else synth.make_grads(w, seed, step)
+        grads = g0 if step == 1 else synth.make_grads(w, seed, step, workers=workers)
         if step > 1:
             for dg, g in zip(dev_g, grads):
                 dg.copy_(to_torch_grad(torch, g, device))
         opt.step(**hp)
-        orc.step([synth.widen(g) for g in grads], **hp)
+        orc.step([synth.widen(grads[i]) for i in sel], **hp)
+        g0 = None
         if step in check_at:
             torch.cuda.synchronize()
-            out[step] = compare_state(opt, orc)
+            out[step] = compare_state(opt, orc, None if oracle_idx is None else sel)
     opt.close()
     return out
