@@ -48,6 +48,22 @@ def dist_env():
         int(os.environ.get("WORLD_SIZE", 1))
 
 
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """Step time of the job: the slowest rank's (all-reduce MAX); identity for one rank."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(world: int, numel_per_rank: int, ms_per_step: float) -> float:
+    """Whole-job throughput: every rank updates its own replica of the parameter set."""
+    return world * numel_per_rank / (ms_per_step * 1e-3)
+
+
 # ---------------------------------------------------------------------------------------
 # clocks
 # ---------------------------------------------------------------------------------------
@@ -176,12 +192,9 @@ def run_gpu(args):
     phase_ms = binding.came_get_phase_ms(opt.ctx)
     phase_names = [binding.came_phase_name(opt.ctx, i) for i in range(len(phase_ms))]
     binding.came_set_profiling(opt.ctx, False)
-    if world > 1:
-        t = torch.tensor([ms], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    ms = max_over_ranks(ms, world, device)
     ms_per_step = ms / args.steps
-    value = world * numel / (ms_per_step * 1e-3)
+    value = job_value(world, numel, ms_per_step)
 
     # ---- end to end: host gradients in, updated parameters out, every step --------------
     e2e = None if args.no_e2e else run_e2e(torch, binding, opt, w, hp, device, world, rank, args)
@@ -293,12 +306,9 @@ def run_e2e(torch, binding, opt, w, hp, device, world, rank, args):
     ev1.record()
     torch.cuda.synchronize()
     ms = ev0.elapsed_time(ev1) / steps
-    if world > 1:
-        tt = torch.tensor([ms], device=device)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        ms = float(tt.item())
+    ms = max_over_ranks(ms, world, device)
     numel = sum(t.numel for t in w.tensors)
-    return {"value": world * numel / (ms * 1e-3), "unit": UNIT, "ms_per_step": ms, "steps": steps,
+    return {"value": job_value(world, numel, ms), "unit": UNIT, "ms_per_step": ms, "steps": steps,
             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
             "api": "came_step_host (pinned host gradients in, updated fp32 parameters out)",
             "host_buffers": "one pinned buffer per distinct shape (host memory budget)" if shared

@@ -1,0 +1,211 @@
+"""GPU tests of the C ABI beyond numerics: error paths that must not launch, resume,
+run-to-run determinism, gradient re-binding, the host-buffer step, queries, profiling and
+guard bands around every buffer (no out-of-bounds write for awkward shapes)."""
+import ctypes
+
+import numpy as np
+import pytest
+
+from paper_2307_02047_b200 import synth
+from tests.parity_util import to_torch_grad
+
+pytestmark = pytest.mark.gpu
+HP = dict(synth.PAPER_HPARAMS)
+GUARD = 64          # floats of sentinel on each side of every buffer
+SENT = 1234.5
+
+
+@pytest.fixture(scope="module")
+def env():
+    import torch
+    from paper_2307_02047_b200 import binding
+    assert torch.cuda.is_available()
+    binding.load()
+    return torch, binding
+
+
+class Buffers:
+    """All tensors of a workload carved out of guarded arenas, as raw descriptors."""
+
+    def __init__(self, torch, binding, w, seed):
+        self.torch, self.w = torch, w
+        self.guards = []
+        self.p, self.g, self.m, self.r, self.c, self.R, self.C = ([] for _ in range(7))
+        params = synth.make_params(w, seed)
+        self.descs = []
+        for i, t in enumerate(w.tensors):
+            p = self._guarded(t.numel, torch.float32); p.copy_(torch.from_numpy(params[i]).reshape(-1))
+            gdt = torch.bfloat16 if w.grad_dtype == synth.BF16 else torch.float32
+            g = self._guarded(t.numel, gdt)
+            m = self._guarded(t.numel, torch.float32)
+            r = self._guarded(t.rows, torch.float32); R = self._guarded(t.rows, torch.float32)
+            c = self._guarded(t.cols, torch.float32) if t.ndim == 2 else None
+            C = self._guarded(t.cols, torch.float32) if t.ndim == 2 else None
+            for lst, x in zip((self.p, self.g, self.m, self.r, self.c, self.R, self.C),
+                              (p, g, m, r, c, R, C)):
+                lst.append(x)
+            ptr = lambda x: x.data_ptr() if x is not None else None
+            self.descs.append(binding.came_tensor(
+                ptr(p), ptr(g), ptr(m), ptr(r), ptr(c), ptr(R), ptr(C), t.rows, t.cols, t.ndim,
+                binding.CAME_BF16 if w.grad_dtype == synth.BF16 else binding.CAME_F32, 0, 0))
+
+    def _guarded(self, n, dtype):
+        torch = self.torch
+        per = 4 // torch.empty(0, dtype=dtype).element_size()      # elements per float slot
+        pad = GUARD * per
+        body = (n + 63) // 64 * 64                                  # keeps the next guard 16-B aligned
+        arena = torch.full((pad + body + pad,), SENT, dtype=dtype, device="cuda:0")
+        self.guards.append((arena, pad, n))
+        return arena[pad:pad + n]
+
+    def set_grads(self, seed, step):
+        for i, g in enumerate(self.g):
+            g.copy_(to_torch_grad(self.torch, synth.make_grad(self.w, seed, i, step), "cuda:0").reshape(-1))
+
+    def check_guards(self):
+        for arena, pad, n in self.guards:
+            a = arena.float().cpu().numpy()
+            assert np.all(a[:pad] == SENT) and np.all(a[pad + n:] == SENT), "guard band overwritten"
+
+    def snapshot(self):
+        self.torch.cuda.synchronize()
+        return [x.clone() for lst in (self.p, self.m, self.r, self.R, self.c, self.C)
+                for x in lst if x is not None]
+
+
+W_ODD = synth.Workload("odd", (synth.mat("a", 257, 1030), synth.mat("b", 33, 65), synth.mat("c", 1, 200),
+                               synth.mat("d", 300, 1), synth.mat("e", 640, 1024), synth.vec("v", 1001),
+                               synth.vec("s", 1)), synth.BF16, "normal_fixed", 1e-3, 0.0, (), 3, HP)
+
+
+def _run_steps(torch, binding, buf, ctx, seed, first, last):
+    stream = torch.cuda.current_stream().cuda_stream
+    for step in range(first, last + 1):
+        buf.set_grads(seed, step)
+        binding.came_step(ctx, binding.make_hparams(step, **HP), None, stream)
+    torch.cuda.synchronize()
+
+
+def _same(a, b):
+    return all(bool((x == y).all()) for x, y in zip(a, b))
+
+
+def test_guard_bands_and_determinism(env):
+    torch, binding = env
+    snaps = []
+    for _ in range(2):
+        buf = Buffers(torch, binding, W_ODD, 3)
+        ctx = binding.came_create(buf.descs)
+        _run_steps(torch, binding, buf, ctx, 3, 1, 3)
+        buf.check_guards()
+        snaps.append(buf.snapshot())
+        binding.came_destroy(ctx)
+    assert _same(*snaps), "two identical runs differ: the reductions are not deterministic"
+
+
+def test_resume_is_bit_exact(env):
+    torch, binding = env
+    a = Buffers(torch, binding, W_ODD, 5)
+    ctx = binding.came_create(a.descs)
+    _run_steps(torch, binding, a, ctx, 5, 1, 6)
+    binding.came_destroy(ctx)
+    b = Buffers(torch, binding, W_ODD, 5)
+    ctx = binding.came_create(b.descs)
+    _run_steps(torch, binding, b, ctx, 5, 1, 3)
+    binding.came_destroy(ctx)
+    ctx = binding.came_create(b.descs, flags=binding.CAME_CREATE_KEEP_STATE)
+    assert binding.came_query(ctx, binding.CAME_Q_LAST_STEP) == 0
+    _run_steps(torch, binding, b, ctx, 5, 4, 6)       # a resumed context accepts any first step
+    binding.came_destroy(ctx)
+    assert _same(a.snapshot(), b.snapshot())
+
+
+def test_errors_do_not_launch(env):
+    torch, binding = env
+    buf = Buffers(torch, binding, W_ODD, 7)
+    ctx = binding.came_create(buf.descs)
+    _run_steps(torch, binding, buf, ctx, 7, 1, 1)
+    before = buf.snapshot()
+    stream = torch.cuda.current_stream().cuda_stream
+    bad = [(dict(HP), 3, 6), (dict(HP), 1, 6), (dict(HP, beta1=1.0), 2, 5), (dict(HP, beta3=-0.1), 2, 5),
+           (dict(HP, clip_d=0.0), 2, 5), (dict(HP, lr=float("nan")), 2, 5), (dict(HP, eps2=-1.0), 2, 5),
+           (dict(HP, weight_decay=-1.0), 2, 5), (dict(HP), 0, 6)]
+    for hp, step, status in bad:
+        with pytest.raises(binding.CameError) as e:
+            binding.came_step(ctx, binding.make_hparams(step, **hp), None, stream)
+        assert e.value.status == status
+    assert _same(before, buf.snapshot())
+    assert binding.came_query(ctx, binding.CAME_Q_LAST_STEP) == 1
+    assert binding.came_last_error(ctx) != ""
+    with pytest.raises(binding.CameError) as e:
+        binding.came_step(ctx, binding.make_hparams(2, **HP), [0] * len(buf.descs), stream)
+    assert e.value.status == 1
+    with pytest.raises(binding.CameError) as e:
+        binding.came_query(ctx, 99)
+    assert e.value.status == 11
+    binding.came_destroy(ctx)
+    with pytest.raises(binding.CameError) as e:
+        binding.came_create(buf.descs, device=4096)
+    assert e.value.status == 7
+
+
+def test_gradient_rebinding_and_host_step(env):
+    torch, binding = env
+    stream = torch.cuda.current_stream().cuda_stream
+    # reference: gradients copied into the buffers given at create
+    a = Buffers(torch, binding, W_ODD, 9)
+    ctx = binding.came_create(a.descs)
+    _run_steps(torch, binding, a, ctx, 9, 1, 3)
+    binding.came_destroy(ctx)
+    # (1) fresh gradient buffers passed to every step
+    b = Buffers(torch, binding, W_ODD, 9)
+    ctx = binding.came_create(b.descs)
+    keep = []
+    for step in (1, 2, 3):
+        gs = [to_torch_grad(torch, synth.make_grad(W_ODD, 9, i, step), "cuda:0").reshape(-1).clone()
+              for i in range(len(W_ODD.tensors))]
+        keep.append(gs)
+        binding.came_step(ctx, binding.make_hparams(step, **HP), [g.data_ptr() for g in gs], stream)
+    torch.cuda.synchronize()
+    binding.came_destroy(ctx)
+    assert _same(a.snapshot(), b.snapshot())
+    # (2) the host-buffer entry point: pinned gradients in, parameters out
+    c = Buffers(torch, binding, W_ODD, 9)
+    ctx = binding.came_create(c.descs)
+    outs = [torch.empty(t.numel, dtype=torch.float32).pin_memory() for t in W_ODD.tensors]
+    for step in (1, 2, 3):
+        hg = [to_torch_grad(torch, synth.make_grad(W_ODD, 9, i, step), "cpu").reshape(-1).pin_memory()
+              for i in range(len(W_ODD.tensors))]
+        binding.came_step_host(ctx, binding.make_hparams(step, **HP), [g.data_ptr() for g in hg],
+                               [o.data_ptr() for o in outs], stream)
+        torch.cuda.synchronize()
+    binding.came_destroy(ctx)
+    assert _same(a.snapshot(), c.snapshot())
+    for o, p in zip(outs, c.p):
+        assert bool((o == p.cpu()).all())
+
+
+def test_queries_and_profiling(env):
+    torch, binding = env
+    w = synth.workload("toy")
+    buf = Buffers(torch, binding, w, 11)
+    ctx = binding.came_create(buf.descs)
+    q = lambda k: binding.came_query(ctx, k)
+    nm, nv = 512 * 256, 256
+    assert q(binding.CAME_Q_NUMEL) == nm + nv
+    assert q(binding.CAME_Q_MATRIX_NUMEL) == nm
+    assert q(binding.CAME_Q_STATE_BYTES) == 4 * (nm + 2 * (512 + 256)) + 12 * nv
+    assert q(binding.CAME_Q_STREAM_BYTES) == nm * 32 + 16 * (512 + 256) + nv * 36
+    assert q(binding.CAME_Q_COMPULSORY_BYTES) == nm * 20 + 16 * (512 + 256) + nv * 36
+    assert q(binding.CAME_Q_LAUNCHES_PER_STEP) == 6 and q(binding.CAME_Q_NUM_PHASES) == 6
+    assert q(binding.CAME_Q_NUM_TILES) >= 1 and q(binding.CAME_Q_WORKSPACE_BYTES) > 0
+    with pytest.raises(binding.CameError):
+        binding.came_get_phase_ms(ctx)                 # nothing profiled yet
+    binding.came_set_profiling(ctx, True)
+    _run_steps(torch, binding, buf, ctx, 11, 1, 4)
+    ms = binding.came_get_phase_ms(ctx)
+    names = [binding.came_phase_name(ctx, i) for i in range(len(ms))]
+    assert names == ["vec_second_moment", "p1_reduce_g2", "p2_sum_u2", "p3_momentum_instability",
+                     "p4_apply", "vec_apply"]
+    assert all(0.0 < x < 50.0 for x in ms)
+    binding.came_destroy(ctx)
