@@ -220,6 +220,8 @@ def run_gpu(args):
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": args.workload, "params": numel,
                    "tensors": len(w.tensors), "grad_dtype": w.grad_dtype,
+                   "tiles": opt.query(binding.CAME_Q_NUM_TILES),
+                   "workspace_bytes": opt.query(binding.CAME_Q_WORKSPACE_BYTES),
                    "state": "fp32 params, m, r, c, R, C",
                    "parallelism": "replicas only" if world > 1 else "single GPU",
                    "l2": "per-step working set %.1f GB >> 126 MB L2; no flush needed"

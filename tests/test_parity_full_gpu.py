@@ -27,8 +27,9 @@ def env(oracle):
     return torch, binding, oracle
 
 
-def _gate(res):
+def _gate(res, label=""):
     assert res
+    print("PARITY", label, {k: {n: float("%.3g" % e) for n, e in v.items()} for k, v in res.items()})
     for step, worst in res.items():
         tol = TOL_STEP1 if step == 1 else TOL_STEP10
         for name, e in worst.items():
@@ -39,7 +40,7 @@ def _gate(res):
 def test_model_shaped_sets_steps_1_and_10(env, name):
     torch, binding, oracle = env
     w = synth.workload(name)
-    _gate(run_paired(torch, binding, oracle, w, seed=2, steps=10, check_at=(1, 10), workers=WORKERS))
+    _gate(run_paired(torch, binding, oracle, w, seed=2, steps=10, check_at=(1, 10), workers=WORKERS), name)
 
 
 def test_bert_large_zero_rows_in_every_matrix(env):
@@ -48,7 +49,7 @@ def test_bert_large_zero_rows_in_every_matrix(env):
     # the oracle follows the embeddings, one layer's matrices and a few vectors
     idx = [0, 1] + list(range(2, 18)) + [1000 % len(w.tensors)]
     _gate(run_paired(torch, binding, oracle, w, seed=4, steps=3, check_at=(1, 3), oracle_idx=idx,
-                     workers=WORKERS))
+                     workers=WORKERS), "bert_large+zero_rows")
 
 
 def test_llama7b_full_set_sampled_tensors(env):
@@ -58,7 +59,7 @@ def test_llama7b_full_set_sampled_tensors(env):
     idx = [names[n] for n in ("tok_emb", "l0.wq", "l0.w_gate", "l0.w_down", "l0.norm1",
                               "l17.wo", "l31.w_up", "l31.norm2", "norm_f")]
     _gate(run_paired(torch, binding, oracle, w, seed=6, steps=2, check_at=(1, 2), oracle_idx=idx,
-                     workers=WORKERS))
+                     workers=WORKERS), "llama7b")
 
 
 @pytest.mark.parametrize("shape", [(1024, 1024), (4096, 4096), (8192, 8192), (16384, 16384),
@@ -68,4 +69,4 @@ def test_shape_sweep_large_matrices(env, shape):
     w = synth.workload(f"mat:{shape[0]}x{shape[1]}")
     steps = 5 if shape[0] * shape[1] <= 1 << 26 else 2
     _gate(run_paired(torch, binding, oracle, w, seed=8, steps=steps, check_at=(1, steps),
-                     workers=WORKERS))
+                     workers=WORKERS), w.name)
