@@ -161,7 +161,9 @@ def run_gpu(args):
     w = synth.workload(args.workload)
     hp = dict(w.hparams)
     params, grads = alloc_device_workload(torch, w, device)
-    opt = binding.CameOptimizer(params, grads, device=local_rank)
+    ada = args.algorithm == "adafactor"
+    opt = binding.CameOptimizer(params, grads, device=local_rank,
+                                create_flags=binding.CAME_CREATE_ADAFACTOR if ada else 0)
     numel = opt.query(binding.CAME_Q_NUMEL)
     stream_bytes = opt.query(binding.CAME_Q_STREAM_BYTES)
     launches = opt.query(binding.CAME_Q_LAUNCHES_PER_STEP)
@@ -201,6 +203,8 @@ def run_gpu(args):
 
     peak, peak_kind = measured_peak()
     pb = phase_bytes(w)
+    pb["p34_adafactor_apply"] = pb["p3_momentum_instability"] + pb["p4_apply"] - 12 * sum(
+        t.numel for t in w.tensors if t.ndim == 2) + 8 * sum(t.numel for t in w.tensors if t.ndim == 2)
     phases = {n: m for n, m in zip(phase_names, phase_ms)}
     matrix_phases = {n: m for n, m in phases.items() if n in pb}
     roofline = None
@@ -218,7 +222,7 @@ def run_gpu(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": {"workload": args.workload, "params": numel,
+        "config": {"workload": args.workload, "algorithm": args.algorithm, "params": numel,
                    "tensors": len(w.tensors), "grad_dtype": w.grad_dtype,
                    "tiles": opt.query(binding.CAME_Q_NUM_TILES),
                    "workspace_bytes": opt.query(binding.CAME_Q_WORKSPACE_BYTES),
@@ -396,6 +400,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--workload", default="llama7b")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--algorithm", default="came", choices=["came", "adafactor"],
+                    help="came = Algorithm 2 (default); adafactor = Algorithm 1, for the cost ratio")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")

@@ -83,7 +83,11 @@ enum {
 
 /* came_create flags */
 enum {
-    CAME_CREATE_KEEP_STATE = 1u << 0     /* resume: do not zero m, r, c, R, C */
+    CAME_CREATE_KEEP_STATE = 1u << 0,    /* resume: do not zero m, r, c, R, C */
+    CAME_CREATE_ADAFACTOR  = 1u << 1     /* run Algorithm 1 (Adafactor with momentum) instead of
+                                            Algorithm 2: the same lines up to m_t, then
+                                            theta_t = theta_{t-1} - eta (m_t + lambda theta_{t-1});
+                                            R and C are not used and may be NULL */
 };
 
 /* One parameter tensor.  All pointers are DEVICE pointers, 16-byte aligned,
@@ -96,6 +100,8 @@ typedef struct {
     float*       c;       /* matrix: fp32 [cols] column factor     | vector: NULL        */
     float*       R;       /* matrix: fp32 [rows] row factor of U   | vector: S [rows]    */
     float*       C;       /* matrix: fp32 [cols] column factor     | vector: NULL        */
+                          /* R (and C) may be NULL where they are not used: Algorithm 1 mode,
+                             or a vector flagged CAME_T_VEC_NO_CONFIDENCE */
     int64_t      rows;    /* >= 1 */
     int64_t      cols;    /* >= 1; must be 1 when ndim == 1 */
     int32_t      ndim;    /* 1 = vector, 2 = matrix; other ranks are not defined by the paper */

@@ -140,7 +140,9 @@ class OracleOptimizer:
     """
 
     def __init__(self, params: Sequence[np.ndarray], no_weight_decay: Sequence[bool] = (),
-                 vec_no_confidence: Sequence[bool] = ()):
+                 vec_no_confidence: Sequence[bool] = (), algorithm: str = "came"):
+        assert algorithm in ("came", "adafactor")   # Algorithm 2 or Algorithm 1
+        self.algorithm = algorithm
         self.p: List[np.ndarray] = [np.ascontiguousarray(x, dtype=np.float64).copy() for x in params]
         self.m = [np.zeros_like(x) for x in self.p]
         self.r, self.c, self.R, self.C = [], [], [], []
@@ -170,7 +172,10 @@ class OracleOptimizer:
         hp = hparams(**kw)
         g = np.ascontiguousarray(g, dtype=np.float64)
         if self.p[i].ndim == 2:
-            matrix_step(self.p[i], g, self.m[i], self.r[i], self.c[i], self.R[i], self.C[i], hp)
+            if self.algorithm == "adafactor":
+                adafactor_matrix_step(self.p[i], g, self.m[i], self.r[i], self.c[i], hp)
+            else:
+                matrix_step(self.p[i], g, self.m[i], self.r[i], self.c[i], self.R[i], self.C[i], hp)
         else:
             vector_step(self.p[i], g, self.m[i], self.r[i], self.R[i], hp,
-                        no_confidence=self.no_conf[i])
+                        no_confidence=self.no_conf[i] or self.algorithm == "adafactor")

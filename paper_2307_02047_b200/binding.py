@@ -20,6 +20,7 @@ CAME_F32, CAME_BF16 = 0, 1
 CAME_T_NO_WEIGHT_DECAY = 1
 CAME_T_VEC_NO_CONFIDENCE = 2
 CAME_CREATE_KEEP_STATE = 1
+CAME_CREATE_ADAFACTOR = 2
 (CAME_Q_NUMEL, CAME_Q_STATE_BYTES, CAME_Q_STREAM_BYTES, CAME_Q_COMPULSORY_BYTES,
  CAME_Q_WORKSPACE_BYTES, CAME_Q_NUM_TILES, CAME_Q_LAUNCHES_PER_STEP, CAME_Q_LAST_STEP,
  CAME_Q_NUM_PHASES, CAME_Q_MATRIX_NUMEL) = range(10)
@@ -209,7 +210,8 @@ class CameOptimizer:
     torch is used for allocation and the stream only.
     """
 
-    def __init__(self, params, grads, flags: Optional[Sequence[int]] = None, device: int = 0):
+    def __init__(self, params, grads, flags: Optional[Sequence[int]] = None, device: int = 0,
+                 create_flags: int = 0):
         import torch
         self.torch = torch
         self.params, self.grads = list(params), list(grads)
@@ -232,7 +234,7 @@ class CameOptimizer:
             descs.append(came_tensor(ptr(p), ptr(g), ptr(self.m[i]), ptr(self.r[i]), ptr(self.c[i]),
                                      ptr(self.R[i]), ptr(self.C[i]), rows, cols, p.dim(), gd,
                                      0 if flags is None else int(flags[i]), 0))
-        self.ctx = came_create(descs, device=device)
+        self.ctx = came_create(descs, device=device, flags=create_flags)
         self.step_count = 0
 
     def step(self, **hp) -> None:

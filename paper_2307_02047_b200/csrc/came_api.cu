@@ -19,11 +19,11 @@ using came::StepConsts;
 
 namespace {
 
-constexpr int kMaxPhases = 6;
+constexpr int kMaxPhases = 7;
 constexpr int kProfSlots = 128;        // profiled steps kept for averaging
 const char* const kPhaseNames[kMaxPhases] = {
     "vec_second_moment", "p1_reduce_g2", "p2_sum_u2", "p3_momentum_instability", "p4_apply",
-    "vec_apply"};
+    "p34_adafactor_apply", "vec_apply"};
 
 thread_local std::string g_create_error;
 long long g_tile_elems_override = 0;   // came_tune(CAME_TUNE_TILE_ELEMS)
@@ -95,6 +95,7 @@ struct came_ctx {
     size_t ws_bytes = 0, table_bytes = 0;
     long long numel = 0, matrix_numel = 0, state_bytes = 0, stream_bytes = 0, comp_bytes = 0;
     long long last_step = 0;
+    bool adafactor = false;                    // Algorithm 1 instead of Algorithm 2
     bool profiling = false;
     std::vector<cudaEvent_t> prof_ev;          // [kProfSlots][kMaxPhases + 1], made on demand
     long long prof_count = 0;                  // profiled steps since profiling was switched on
@@ -119,7 +120,7 @@ came_status cuda_fail(came_ctx* ctx, cudaError_t e, const char* what)
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
-came_status validate_tensor(const came_tensor& t, int i, std::string& msg)
+came_status validate_tensor(const came_tensor& t, int i, bool adafactor, std::string& msg)
 {
     char buf[160];
     auto err = [&](came_status s, const char* what) {
@@ -133,8 +134,12 @@ came_status validate_tensor(const came_tensor& t, int i, std::string& msg)
     if (t.rows > (1ll << 40) / t.cols) return err(CAME_ERR_SHAPE, "tensor too large");
     if (t.grad_dtype != CAME_F32 && t.grad_dtype != CAME_BF16) return err(CAME_ERR_DTYPE, "unknown grad_dtype");
     if (t.reserved != 0) return err(CAME_ERR_SHAPE, "reserved must be 0");
-    if (!t.param || !t.grad || !t.m || !t.r || !t.R) return err(CAME_ERR_NULL, "param, grad, m, r, R are required");
-    if (t.ndim == 2 && (!t.c || !t.C)) return err(CAME_ERR_NULL, "a matrix needs c and C");
+    if (!t.param || !t.grad || !t.m || !t.r) return err(CAME_ERR_NULL, "param, grad, m, r are required");
+    if (t.ndim == 2 && !t.c) return err(CAME_ERR_NULL, "a matrix needs c");
+    if (!adafactor && !(t.ndim == 1 && (t.flags & CAME_T_VEC_NO_CONFIDENCE))) {
+        if (!t.R) return err(CAME_ERR_NULL, "R is required");
+        if (t.ndim == 2 && !t.C) return err(CAME_ERR_NULL, "a matrix needs C");
+    }
     const void* ptrs[7] = {t.param, t.grad, t.m, t.r, t.c, t.R, t.C};
     for (const void* p : ptrs)
         if (p && !aligned(p, 16)) return err(CAME_ERR_ALIGN, "pointer not 16-byte aligned");
@@ -239,12 +244,18 @@ came_status launch_step(came_ctx* ctx, const came_hparams* hp, cudaStream_t stre
         came::k_p2_sum_u2<<<ctx->n_tiles, came::kThreads, 0, stream>>>(
             ctx->d_table, ctx->d_tiles, ctx->n_tiles, 1, hc);
         mark(++iv);
-        came::k_p3_momentum_instability<<<ctx->n_tiles, came::kThreads, 0, stream>>>(
-            ctx->d_table, ctx->d_tiles, ctx->n_tiles, 0, hc);
-        mark(++iv);
-        came::k_p4_apply<<<ctx->n_tiles, came::kThreads, 0, stream>>>(
-            ctx->d_table, ctx->d_tiles, ctx->n_tiles, 1, hc);
-        mark(++iv);
+        if (ctx->adafactor) {
+            came::k_p34_adafactor_apply<<<ctx->n_tiles, came::kThreads, 0, stream>>>(
+                ctx->d_table, ctx->d_tiles, ctx->n_tiles, 0, hc);
+            mark(++iv);
+        } else {
+            came::k_p3_momentum_instability<<<ctx->n_tiles, came::kThreads, 0, stream>>>(
+                ctx->d_table, ctx->d_tiles, ctx->n_tiles, 0, hc);
+            mark(++iv);
+            came::k_p4_apply<<<ctx->n_tiles, came::kThreads, 0, stream>>>(
+                ctx->d_table, ctx->d_tiles, ctx->n_tiles, 1, hc);
+            mark(++iv);
+        }
     }
     if (ctx->n_chunks > 0) {
         came::k_vec_apply<<<ctx->n_chunks, came::kThreads, 0, stream>>>(
@@ -314,11 +325,12 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
     *out = nullptr;
     if (!t) return fail(nullptr, CAME_ERR_NULL, "tensor array is NULL");
     if (n < 1) return fail(nullptr, CAME_ERR_SHAPE, "need at least one tensor");
-    if (flags & ~static_cast<uint32_t>(CAME_CREATE_KEEP_STATE))
+    if (flags & ~static_cast<uint32_t>(CAME_CREATE_KEEP_STATE | CAME_CREATE_ADAFACTOR))
         return fail(nullptr, CAME_ERR_UNSUPPORTED, "unknown create flag");
+    const bool adafactor = (flags & CAME_CREATE_ADAFACTOR) != 0;
     std::string msg;
     for (int i = 0; i < n; ++i) {
-        const came_status s = validate_tensor(t[i], i, msg);
+        const came_status s = validate_tensor(t[i], i, adafactor, msg);
         if (s != CAME_OK) return fail(nullptr, s, msg);
     }
     int ndev = 0;
@@ -333,6 +345,7 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
     came_ctx* ctx = new (std::nothrow) came_ctx;
     if (!ctx) return fail(nullptr, CAME_ERR_OOM, "host allocation failed");
     ctx->device = device;
+    ctx->adafactor = adafactor;
     ctx->n = n;
     ctx->tensors.assign(t, t + n);
     ctx->host_table.resize(n);
@@ -364,9 +377,15 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
         ctx->numel += numel;
         if (x.ndim == 2) {
             ctx->matrix_numel += numel;
-            ctx->state_bytes += 4 * (numel + 2 * (x.rows + x.cols));
-            ctx->stream_bytes += numel * (3 * sg + 20) + 16 * (x.rows + x.cols);
-            ctx->comp_bytes += numel * (sg + 16) + 16 * (x.rows + x.cols);
+            if (adafactor) {
+                ctx->state_bytes += 4 * (numel + (x.rows + x.cols));
+                ctx->stream_bytes += numel * (3 * sg + 16) + 8 * (x.rows + x.cols);
+                ctx->comp_bytes += numel * (sg + 16) + 8 * (x.rows + x.cols);
+            } else {
+                ctx->state_bytes += 4 * (numel + 2 * (x.rows + x.cols));
+                ctx->stream_bytes += numel * (3 * sg + 20) + 16 * (x.rows + x.cols);
+                ctx->comp_bytes += numel * (sg + 16) + 16 * (x.rows + x.cols);
+            }
             for (int rb = 0; rb < p.n_rb; ++rb)
                 for (int cb = 0; cb < p.n_cb; ++cb) tiles.push_back(Tile{i, rb, cb});
             offs[i].colpart = take(sizeof(float) * static_cast<size_t>(p.n_rb) * x.cols);
@@ -375,9 +394,10 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
             offs[i].rowscale = take(sizeof(float) * static_cast<size_t>(x.rows));
             offs[i].colscale = take(sizeof(float) * static_cast<size_t>(x.cols));
         } else {
-            ctx->state_bytes += 4 * 3 * numel;
-            ctx->stream_bytes += numel * (sg + 32);
-            ctx->comp_bytes += numel * (sg + 32);
+            const bool conf = !adafactor && !(x.flags & CAME_T_VEC_NO_CONFIDENCE);
+            ctx->state_bytes += 4 * (conf ? 3 : 2) * numel;
+            ctx->stream_bytes += numel * (sg + (conf ? 32 : 24));
+            ctx->comp_bytes += numel * (sg + (conf ? 32 : 24));
             for (int c = 0; c < p.n_parts; ++c) chunks.push_back(VChunk{i, c});
             offs[i].colpart = offs[i].rowpart = offs[i].blocksum = 0;
             offs[i].rowscale = offs[i].colscale = 0;
@@ -436,14 +456,15 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
         int lg = 0; while ((1 << lg) < p.tx) ++lg;
         d.tx_log2 = lg; d.tr = p.tr; d.n_rb = p.n_rb; d.n_cb = p.n_cb; d.n_seg = p.n_seg;
         d.n_parts = p.n_parts; d.ndim = x.ndim; d.flags = x.flags;
+        if (adafactor && x.ndim == 1) d.flags |= came::kFlagVecNoConf;   // Algorithm 1 has no S
         if (!(flags & CAME_CREATE_KEEP_STATE)) {
             const size_t numel = static_cast<size_t>(x.rows) * x.cols;
             CAME_TRY(cudaMemsetAsync(x.m, 0, 4 * numel, 0), "cudaMemset(m)");
             CAME_TRY(cudaMemsetAsync(x.r, 0, 4 * static_cast<size_t>(x.rows), 0), "cudaMemset(r)");
-            CAME_TRY(cudaMemsetAsync(x.R, 0, 4 * static_cast<size_t>(x.rows), 0), "cudaMemset(R)");
+            if (x.R) CAME_TRY(cudaMemsetAsync(x.R, 0, 4 * static_cast<size_t>(x.rows), 0), "cudaMemset(R)");
             if (x.ndim == 2) {
                 CAME_TRY(cudaMemsetAsync(x.c, 0, 4 * static_cast<size_t>(x.cols), 0), "cudaMemset(c)");
-                CAME_TRY(cudaMemsetAsync(x.C, 0, 4 * static_cast<size_t>(x.cols), 0), "cudaMemset(C)");
+                if (x.C) CAME_TRY(cudaMemsetAsync(x.C, 0, 4 * static_cast<size_t>(x.cols), 0), "cudaMemset(C)");
             }
         }
     }
@@ -533,9 +554,11 @@ came_status came_query(const came_ctx* ctx, int32_t what, int64_t* out)
                                         sizeof(VChunk) * ctx->n_chunks);
             break;
         case CAME_Q_NUM_TILES: *out = ctx->n_tiles; break;
-        case CAME_Q_LAUNCHES_PER_STEP: *out = (ctx->n_tiles ? 4 : 0) + (ctx->n_chunks ? 2 : 0); break;
+        case CAME_Q_LAUNCHES_PER_STEP:
+            *out = (ctx->n_tiles ? (ctx->adafactor ? 3 : 4) : 0) + (ctx->n_chunks ? 2 : 0); break;
         case CAME_Q_LAST_STEP: *out = ctx->last_step; break;
-        case CAME_Q_NUM_PHASES: *out = (ctx->n_tiles ? 4 : 0) + (ctx->n_chunks ? 2 : 0); break;
+        case CAME_Q_NUM_PHASES:
+            *out = (ctx->n_tiles ? (ctx->adafactor ? 3 : 4) : 0) + (ctx->n_chunks ? 2 : 0); break;
         case CAME_Q_MATRIX_NUMEL: *out = ctx->matrix_numel; break;
         default: return CAME_ERR_UNSUPPORTED;
     }
@@ -588,8 +611,9 @@ const char* came_phase_name(const came_ctx* ctx, int32_t phase)
     if (!ctx || phase < 0) return "";
     // phases are reported in launch order; vectors-only or matrices-only contexts skip some
     int idx = 0;
-    const bool has[kMaxPhases] = {ctx->n_chunks > 0, ctx->n_tiles > 0, ctx->n_tiles > 0,
-                                  ctx->n_tiles > 0, ctx->n_tiles > 0, ctx->n_chunks > 0};
+    const bool mat = ctx->n_tiles > 0, ada = ctx->adafactor;
+    const bool has[kMaxPhases] = {ctx->n_chunks > 0, mat, mat, mat && !ada, mat && !ada, mat && ada,
+                                  ctx->n_chunks > 0};
     for (int k = 0; k < kMaxPhases; ++k) {
         if (!has[k]) continue;
         if (idx == phase) return kPhaseNames[k];

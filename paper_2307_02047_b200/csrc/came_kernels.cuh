@@ -658,6 +658,69 @@ __device__ __forceinline__ void p4_tile(const TensorDev& d, int rb, int cb, cons
 }
 
 // ---------------------------------------------------------------------------
+// Algorithm 1 (Adafactor with momentum), the lines after the clip: with kappa known there is
+// no further tensor-wide dependency, so momentum and parameter update are one pass:
+//   m_t = m_{t-1} + (1-beta1)(uhat_t - m_{t-1});  theta -= lr * (m_t + wd * theta)
+// ---------------------------------------------------------------------------
+template <int KIND>
+__device__ __forceinline__ void p34_adafactor_tile(const TensorDev& d, int rb, int cb,
+                                                   const StepConsts& hc)
+{
+    constexpr int VEC = Traits<KIND>::VEC;
+    constexpr int U = CAME_P34_U;
+    const Geo q = make_geo<VEC>(d, rb, cb);
+    if (!q.colok) return;
+    const long long first = (q.row0 + q.ty) * d.cols + q.col;
+    const long long gstride = static_cast<long long>(q.TY) * d.cols * grad_elem_bytes<KIND>();
+    const long long stride = static_cast<long long>(q.TY) * d.cols;
+    const char* gp = static_cast<const char*>(d.g) + first * grad_elem_bytes<KIND>();
+    float* mp = d.m + first;
+    float* pp = d.p + first;
+    const float* ap = d.ws_rowscale + q.row0 + q.ty;
+    const float ssr_k = d.scal[0] * d.scal[1];
+    const float wd = (d.flags & kFlagNoWd) ? 0.f : hc.wd;
+    const float nlr = -hc.lr, omb1 = hc.omb1;
+    float b[VEC];
+#pragma unroll
+    for (int v = 0; v < VEC; ++v) b[v] = d.ws_colscale[q.col + v];
+
+    for (long long rbase = q.row0 + q.ty; rbase < q.row1; rbase += static_cast<long long>(q.TY) * U) {
+        Raw<KIND> raw[U];
+        float mo[U][VEC], th[U][VEC], a[U];
+        const bool full = rbase + static_cast<long long>(U - 1) * q.TY < q.row1;
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            if (full || rbase + static_cast<long long>(k) * q.TY < q.row1) {
+                load_raw<KIND>(gp + k * gstride, raw[k]);
+                load_f<VEC>(mp + k * stride, mo[k]);
+                load_f<VEC>(pp + k * stride, th[k]);
+                a[k] = ap[k * q.TY];
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < U; ++k) {
+            if (full || rbase + static_cast<long long>(k) * q.TY < q.row1) {
+                float x[VEC];
+                unpack<KIND>(raw[k], x);
+                const float ai = a[k] * ssr_k;
+#pragma unroll
+                for (int v = 0; v < VEC; ++v) {
+                    const float uh = (x[v] * b[v]) * ai;
+                    mo[k][v] = fmaf(omb1, uh - mo[k][v], mo[k][v]);
+                    th[k][v] = fmaf(nlr, fmaf(wd, th[k][v], mo[k][v]), th[k][v]);
+                }
+                store_f<VEC>(mp + k * stride, mo[k]);
+                store_f<VEC>(pp + k * stride, th[k]);
+            }
+        }
+        gp += U * gstride;
+        mp += U * stride;
+        pp += U * stride;
+        ap += U * q.TY;
+    }
+}
+
+// ---------------------------------------------------------------------------
 // kernels: one block per tile, block-uniform dispatch on the tensor's kind
 // ---------------------------------------------------------------------------
 #define CAME_DISPATCH(FN, ...)                                         \
@@ -711,6 +774,15 @@ k_p4_apply(const TensorDev* __restrict__ T, const Tile* __restrict__ tiles, int 
     const Tile t = fetch_tile(tiles, ntiles, reverse);
     const TensorDev d = T[t.tensor];
     CAME_DISPATCH(p4_tile, d, t.rb, t.cb, hc)
+}
+
+__global__ void __launch_bounds__(kThreads, 2)
+k_p34_adafactor_apply(const TensorDev* __restrict__ T, const Tile* __restrict__ tiles, int ntiles,
+                      int reverse, StepConsts hc)
+{
+    const Tile t = fetch_tile(tiles, ntiles, reverse);
+    const TensorDev d = T[t.tensor];
+    CAME_DISPATCH(p34_adafactor_tile, d, t.rb, t.cb, hc)
 }
 
 // ---------------------------------------------------------------------------

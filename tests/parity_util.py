@@ -58,7 +58,8 @@ def compare_state(opt, orc, indices=None) -> dict:
 
 
 def run_paired(torch, binding, oracle, w: synth.Workload, seed: int, steps: int, check_at,
-               flags=None, hparams=None, device="cuda:0", oracle_idx=None, workers: int = 0):
+               flags=None, hparams=None, device="cuda:0", oracle_idx=None, workers: int = 0,
+               algorithm: str = "came"):
     """Step the CUDA path and the oracle side by side; returns {step: worst-error dict}.
 
     ``oracle_idx``: run the oracle on these tensors only (tensors are independent, so each is
@@ -69,12 +70,13 @@ def run_paired(torch, binding, oracle, w: synth.Workload, seed: int, steps: int,
     dev_p = [torch.from_numpy(p).to(device) for p in params]
     g0 = synth.make_grads(w, seed, 1, workers=workers)
     dev_g = [to_torch_grad(torch, g, device) for g in g0]
-    opt = binding.CameOptimizer(dev_p, dev_g, flags=flags)
+    opt = binding.CameOptimizer(dev_p, dev_g, flags=flags,
+                                create_flags=binding.CAME_CREATE_ADAFACTOR if algorithm == "adafactor" else 0)
     sel = list(range(len(params))) if oracle_idx is None else list(oracle_idx)
     no_wd = [bool(flags[i] & binding.CAME_T_NO_WEIGHT_DECAY) for i in sel] if flags else ()
     no_conf = [bool(flags[i] & binding.CAME_T_VEC_NO_CONFIDENCE) for i in sel] if flags else ()
     orc = oracle.OracleOptimizer([params[i] for i in sel], no_weight_decay=no_wd,
-                                 vec_no_confidence=no_conf)
+                                 vec_no_confidence=no_conf, algorithm=algorithm)
     del params
     out = {}
     for step in range(1, steps + 1):

@@ -70,3 +70,10 @@ def test_shape_sweep_large_matrices(env, shape):
     steps = 5 if shape[0] * shape[1] <= 1 << 26 else 2
     _gate(run_paired(torch, binding, oracle, w, seed=8, steps=steps, check_at=(1, steps),
                      workers=WORKERS), w.name)
+
+
+def test_bert_base_adafactor_mode(env):
+    torch, binding, oracle = env
+    w = synth.workload("bert_base")
+    _gate(run_paired(torch, binding, oracle, w, seed=2, steps=10, check_at=(1, 10), workers=WORKERS,
+                     algorithm="adafactor"), "bert_base/adafactor")

@@ -90,3 +90,44 @@ def test_other_hyperparameters(env):
     hp0 = dict(synth.PAPER_HPARAMS, beta1=0.0, clip_d=100.0)
     _gate(run_paired(torch, binding, oracle, synth.workload("toy"), seed=13, steps=3,
                      check_at=(1, 3), hparams=hp0))
+
+
+# ---------------------------------------------------------------------------
+# Algorithm 1 (Adafactor with momentum) on the same kernels
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("name", ["toy", "mat:257x1030:bf16", "mat:1x4096", "mat:777x768"])
+def test_adafactor_mode(env, name):
+    torch, binding, oracle = env
+    w = synth.workload(name)
+    hp = dict(w.hparams, weight_decay=0.01)
+    _gate(run_paired(torch, binding, oracle, w, seed=17, steps=10, check_at=(1, 10), hparams=hp,
+                     algorithm="adafactor"))
+
+
+def test_adafactor_mode_needs_no_instability_state(env):
+    torch, binding, oracle = env
+    w = synth.workload("toy")
+    params = synth.make_params(w, 19)
+    p = [torch.from_numpy(x).cuda() for x in params]
+    g = [torch.from_numpy(x).cuda() for x in synth.make_grads(w, 19, 1)]
+    m = [torch.empty_like(x) for x in p]
+    r = [torch.empty(512, device="cuda"), torch.empty(256, device="cuda")]
+    c = torch.empty(256, device="cuda")
+    descs = [binding.came_tensor(p[0].data_ptr(), g[0].data_ptr(), m[0].data_ptr(), r[0].data_ptr(),
+                                 c.data_ptr(), None, None, 512, 256, 2, 0, 0, 0),
+             binding.came_tensor(p[1].data_ptr(), g[1].data_ptr(), m[1].data_ptr(), r[1].data_ptr(),
+                                 None, None, None, 256, 1, 1, 0, 0, 0)]
+    with pytest.raises(binding.CameError) as e:
+        binding.came_create(descs)                      # Algorithm 2 needs R and C
+    assert e.value.status == 1
+    ctx = binding.came_create(descs, flags=binding.CAME_CREATE_ADAFACTOR)
+    assert binding.came_query(ctx, binding.CAME_Q_LAUNCHES_PER_STEP) == 5
+    binding.came_step(ctx, binding.make_hparams(1, **w.hparams), None,
+                      torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    orc = oracle.OracleOptimizer(params, algorithm="adafactor")
+    orc.step([synth.widen(x) for x in synth.make_grads(w, 19, 1)], **w.hparams)
+    from tests.parity_util import err_signed
+    assert err_signed(p[0].cpu().numpy(), orc.p[0]) <= TOL_STEP1
+    assert err_signed(p[1].cpu().numpy(), orc.p[1]) <= TOL_STEP1
+    binding.came_destroy(ctx)
