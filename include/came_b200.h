@@ -108,6 +108,10 @@ typedef struct {
     int32_t      grad_dtype;  /* came_dtype */
     uint32_t     flags;   /* CAME_T_* */
     uint32_t     reserved;    /* must be 0 */
+    void*        param_bf16;  /* optional DEVICE bf16 [rows*cols], 16-byte aligned: receives the
+                                 updated parameters rounded to nearest-even bf16 in the same pass
+                                 that writes `param` (the copy the next forward pass reads);
+                                 NULL = none.  Not part of the paper's algorithm. */
 } came_tensor;
 
 /* Hyper-parameters of one step (doubles: 1-beta is formed in double, then each
@@ -123,6 +127,9 @@ typedef struct {
     double  weight_decay;  /* lambda >= 0 (extension; 0 = the paper)        */
     int64_t step;          /* t >= 1; must be previous + 1 after the first call.  Not used
                               in the arithmetic (Algorithm 2 has no bias correction). */
+    double  grad_scale;    /* s > 0: the step uses g_t = s * (gradient buffer), e.g. 1/(number of
+                              accumulation steps) or 1/(loss scale); 0 means 1.  Folded into the
+                              per-tensor scalars, so it costs no pass and no per-element work. */
 } came_hparams;
 
 /* came_query selectors */

@@ -42,14 +42,15 @@ class came_tensor(ctypes.Structure):
                 ("r", ctypes.c_void_p), ("c", ctypes.c_void_p), ("R", ctypes.c_void_p),
                 ("C", ctypes.c_void_p), ("rows", ctypes.c_int64), ("cols", ctypes.c_int64),
                 ("ndim", ctypes.c_int32), ("grad_dtype", ctypes.c_int32),
-                ("flags", ctypes.c_uint32), ("reserved", ctypes.c_uint32)]
+                ("flags", ctypes.c_uint32), ("reserved", ctypes.c_uint32),
+                ("param_bf16", ctypes.c_void_p)]
 
 
 class came_hparams(ctypes.Structure):
     _fields_ = [("lr", ctypes.c_double), ("beta1", ctypes.c_double), ("beta2", ctypes.c_double),
                 ("beta3", ctypes.c_double), ("eps1", ctypes.c_double), ("eps2", ctypes.c_double),
                 ("clip_d", ctypes.c_double), ("weight_decay", ctypes.c_double),
-                ("step", ctypes.c_int64)]
+                ("step", ctypes.c_int64), ("grad_scale", ctypes.c_double)]
 
 
 _lib = None
@@ -196,7 +197,8 @@ def came_factor_update_static(grad: int, grad_dtype: int, rows: int, cols: int, 
 def make_hparams(step: int, **kw) -> came_hparams:
     return came_hparams(float(kw["lr"]), float(kw["beta1"]), float(kw["beta2"]), float(kw["beta3"]),
                         float(kw["eps1"]), float(kw["eps2"]), float(kw["clip_d"]),
-                        float(kw.get("weight_decay", 0.0)), int(step))
+                        float(kw.get("weight_decay", 0.0)), int(step),
+                        float(kw.get("grad_scale", 1.0)))
 
 
 # --- convenience wrapper -------------------------------------------------------------------
@@ -211,11 +213,12 @@ class CameOptimizer:
     """
 
     def __init__(self, params, grads, flags: Optional[Sequence[int]] = None, device: int = 0,
-                 create_flags: int = 0):
+                 create_flags: int = 0, bf16_copy: bool = False):
         import torch
         self.torch = torch
         self.params, self.grads = list(params), list(grads)
         self.m, self.r, self.c, self.R, self.C = [], [], [], [], []
+        self.p_bf16 = []
         descs = []
         for i, (p, g) in enumerate(zip(self.params, self.grads)):
             assert p.is_cuda and p.dtype == torch.float32 and p.is_contiguous()
@@ -231,9 +234,10 @@ class CameOptimizer:
             gd = CAME_BF16 if g.dtype == torch.bfloat16 else CAME_F32
             assert g.dtype in (torch.bfloat16, torch.float32)
             ptr = lambda t: t.data_ptr() if t is not None else None
+            self.p_bf16.append(torch.empty_like(p, dtype=torch.bfloat16) if bf16_copy else None)
             descs.append(came_tensor(ptr(p), ptr(g), ptr(self.m[i]), ptr(self.r[i]), ptr(self.c[i]),
                                      ptr(self.R[i]), ptr(self.C[i]), rows, cols, p.dim(), gd,
-                                     0 if flags is None else int(flags[i]), 0))
+                                     0 if flags is None else int(flags[i]), 0, ptr(self.p_bf16[i])))
         self.ctx = came_create(descs, device=device, flags=create_flags)
         self.step_count = 0
 

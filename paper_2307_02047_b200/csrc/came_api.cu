@@ -140,7 +140,7 @@ came_status validate_tensor(const came_tensor& t, int i, bool adafactor, std::st
         if (!t.R) return err(CAME_ERR_NULL, "R is required");
         if (t.ndim == 2 && !t.C) return err(CAME_ERR_NULL, "a matrix needs C");
     }
-    const void* ptrs[7] = {t.param, t.grad, t.m, t.r, t.c, t.R, t.C};
+    const void* ptrs[8] = {t.param, t.grad, t.m, t.r, t.c, t.R, t.C, t.param_bf16};
     for (const void* p : ptrs)
         if (p && !aligned(p, 16)) return err(CAME_ERR_ALIGN, "pointer not 16-byte aligned");
     if ((t.flags & CAME_T_VEC_NO_CONFIDENCE) && t.ndim != 1)
@@ -150,7 +150,8 @@ came_status validate_tensor(const came_tensor& t, int i, bool adafactor, std::st
 
 came_status validate_hparams(const came_hparams& h, long long last_step, std::string& msg)
 {
-    const double v[8] = {h.lr, h.beta1, h.beta2, h.beta3, h.eps1, h.eps2, h.clip_d, h.weight_decay};
+    const double v[9] = {h.lr, h.beta1, h.beta2, h.beta3, h.eps1, h.eps2, h.clip_d, h.weight_decay,
+                         h.grad_scale};
     for (double x : v)
         if (!std::isfinite(x)) { msg = "hyper-parameter not finite"; return CAME_ERR_HPARAM; }
     if (h.lr < 0) { msg = "lr must be >= 0"; return CAME_ERR_HPARAM; }
@@ -160,6 +161,7 @@ came_status validate_hparams(const came_hparams& h, long long last_step, std::st
     if (h.eps1 < 0 || h.eps2 < 0) { msg = "eps1, eps2 must be >= 0"; return CAME_ERR_HPARAM; }
     if (!(h.clip_d > 0)) { msg = "clip_d must be > 0"; return CAME_ERR_HPARAM; }
     if (h.weight_decay < 0) { msg = "weight_decay must be >= 0"; return CAME_ERR_HPARAM; }
+    if (h.grad_scale < 0) { msg = "grad_scale must be > 0 (or 0 for 1)"; return CAME_ERR_HPARAM; }
     if (h.step < 1) { msg = "step must be >= 1"; return CAME_ERR_STEP_ORDER; }
     if (last_step > 0 && h.step != last_step + 1) {
         msg = "step must be the previous step + 1";
@@ -182,6 +184,9 @@ StepConsts make_consts(const came_hparams& h)
     c.eps2 = static_cast<float>(h.eps2);
     c.lr = static_cast<float>(h.lr);
     c.wd = static_cast<float>(h.weight_decay);
+    const double gs = h.grad_scale == 0.0 ? 1.0 : h.grad_scale;
+    c.gscale = static_cast<float>(gs);
+    c.gscale2 = static_cast<float>(gs * gs);
     c.pad_ = 0.f;
     c.clip_d = h.clip_d;
     return c;
@@ -375,6 +380,7 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
         const long long numel = x.rows * x.cols;
         const long long sg = x.grad_dtype == CAME_BF16 ? 2 : 4;
         ctx->numel += numel;
+        if (x.param_bf16) { ctx->stream_bytes += 2 * numel; ctx->comp_bytes += 2 * numel; }
         if (x.ndim == 2) {
             ctx->matrix_numel += numel;
             if (adafactor) {
@@ -443,6 +449,7 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
         TensorDev& d = ctx->host_table[i];
         std::memset(&d, 0, sizeof d);
         d.p = x.param; d.g = x.grad; d.m = x.m; d.r = x.r; d.c = x.c; d.R = x.R; d.C = x.C;
+        d.p_bf16 = static_cast<uint16_t*>(x.param_bf16);
         d.rows = x.rows; d.cols = x.cols;
         d.ws_colpart = reinterpret_cast<float*>(ctx->d_ws + offs[i].colpart);
         d.ws_rowpart = reinterpret_cast<float*>(ctx->d_ws + offs[i].rowpart);
@@ -735,6 +742,8 @@ extern "C" came_status came_factor_update_static(const void* grad, int32_t grad_
     hc.beta2 = static_cast<float>(beta2);
     hc.omb2 = static_cast<float>(1.0 - beta2);
     hc.eps1 = static_cast<float>(eps1);
+    hc.gscale = 1.f;
+    hc.gscale2 = 1.f;
     hc.clip_d = 1.0;
     k_p1_reduce_g2_single<<<p.n_rb * p.n_cb, came::kThreads, 0, stream>>>(d, hc);
     e = cudaGetLastError();

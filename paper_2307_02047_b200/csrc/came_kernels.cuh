@@ -64,6 +64,7 @@ struct TensorDev {
     float*       ws_colscale;  // [cols]  rsqrt of the column factor last finished (c_t, then C_t)
     unsigned*    cnt;          // [n_rb] row-block arrivals, [n_cb] strip arrivals, [1] finished, [1] usq
     float*       scal;         // [0] sqrt(sum r)  [1] kappa  [2] sqrt(sum R)
+    uint16_t*    p_bf16;       // optional bf16 copy of the updated parameters (NULL = none)
     int          kind;
     int          vec;          // elements per thread per load
     int          tx_log2;      // threads across columns = 1 << tx_log2 (32..256)
@@ -83,6 +84,7 @@ struct StepConsts {
     float beta3, omb3;
     float eps1, eps2;
     float lr, wd;
+    float gscale, gscale2;   // gradient pre-scale s and s^2 (g_t = s * gradient buffer)
     float pad_;
     double clip_d;
 };
@@ -130,6 +132,32 @@ __device__ __forceinline__ void store_f(float* p, const float (&x)[VEC])
                      :: "l"(p), "f"(x[0]), "f"(x[1]), "f"(x[2]), "f"(x[3]) : "memory");
     } else {
         *p = x[0];
+    }
+}
+
+// two fp32 -> packed bf16x2, round to nearest even (lo in the low half)
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    uint32_t r;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo));
+    return r;
+}
+
+// bf16 copy of VEC consecutive fp32 values (VEC = 8: one 128-bit store, 4: 64-bit, 1: 16-bit)
+template <int VEC>
+__device__ __forceinline__ void store_bf16(uint16_t* p, const float (&x)[VEC])
+{
+    if constexpr (VEC == 8) {
+        uint4 v;
+        v.x = pack_bf16x2(x[0], x[1]); v.y = pack_bf16x2(x[2], x[3]);
+        v.z = pack_bf16x2(x[4], x[5]); v.w = pack_bf16x2(x[6], x[7]);
+        *reinterpret_cast<uint4*>(p) = v;
+    } else if constexpr (VEC == 4) {
+        uint2 v;
+        v.x = pack_bf16x2(x[0], x[1]); v.y = pack_bf16x2(x[2], x[3]);
+        *reinterpret_cast<uint2*>(p) = v;
+    } else {
+        *p = static_cast<uint16_t>(pack_bf16x2(x[0], 0.f) & 0xffffu);
     }
 }
 
@@ -466,7 +494,7 @@ __device__ __forceinline__ void p1_tile(const TensorDev& d, int rb, int cb, cons
         store_row_partials<U>(rs, rowpart_seg, rbase, q.TY, q.row1, lane);
     }
     write_col_partials<VEC>(d, q, rb, cacc, sm);
-    finalize_factors(d, rb, cb, hc.beta2, hc.omb2, hc.eps1, 1.0f, d.r, d.c, d.scal + 0, sm);
+    finalize_factors(d, rb, cb, hc.beta2, hc.omb2, hc.eps1, hc.gscale2, d.r, d.c, d.scal + 0, sm);
 }
 
 // ---------------------------------------------------------------------------
@@ -483,7 +511,7 @@ __device__ __forceinline__ void p2_tile(const TensorDev& d, int rb, int cb, cons
     const char* gp = static_cast<const char*>(d.g) +
                      ((q.row0 + q.ty) * d.cols + q.col) * grad_elem_bytes<KIND>();
     const float* ap = d.ws_rowscale + q.row0 + q.ty;
-    const float ssr = d.scal[0];
+    const float ssr = d.scal[0] * hc.gscale;          // sqrt(sum r) * gradient pre-scale
     float b[VEC];
 #pragma unroll
     for (int v = 0; v < VEC; ++v) b[v] = q.colok ? d.ws_colscale[q.col + v] : 0.f;
@@ -542,7 +570,7 @@ __device__ __forceinline__ void p3_tile(const TensorDev& d, int rb, int cb, cons
     float* mp = d.m + first;
     const float* ap = d.ws_rowscale + q.row0 + q.ty;
     float* const rowpart_seg = d.ws_rowpart + q.seg * d.rows;
-    const float ssr_k = d.scal[0] * d.scal[1];          // sqrt(sum r) * kappa
+    const float ssr_k = d.scal[0] * d.scal[1] * hc.gscale;   // sqrt(sum r) * kappa * pre-scale
     const float omb1 = hc.omb1;
     float b[VEC], cacc[VEC];
 #pragma unroll
@@ -620,6 +648,7 @@ __device__ __forceinline__ void p4_tile(const TensorDev& d, int rb, int cb, cons
     const long long stride = static_cast<long long>(q.TY) * d.cols;
     const float* mp = d.m + first;
     float* pp = d.p + first;
+    uint16_t* hp16 = d.p_bf16 ? d.p_bf16 + first : nullptr;
     const float* ap = d.ws_rowscale + q.row0 + q.ty;
     const float ssR = d.scal[2];
     const float wd = (d.flags & kFlagNoWd) ? 0.f : hc.wd;
@@ -649,10 +678,12 @@ __device__ __forceinline__ void p4_tile(const TensorDev& d, int rb, int cb, cons
                     th[k][v] = fmaf(nlr, upd, th[k][v]);
                 }
                 store_f<VEC>(pp + k * stride, th[k]);
+                if (hp16) store_bf16<VEC>(hp16 + k * stride, th[k]);
             }
         }
         mp += U * stride;
         pp += U * stride;
+        if (hp16) hp16 += U * stride;
         ap += U * q.TY;
     }
 }
@@ -676,8 +707,9 @@ __device__ __forceinline__ void p34_adafactor_tile(const TensorDev& d, int rb, i
     const char* gp = static_cast<const char*>(d.g) + first * grad_elem_bytes<KIND>();
     float* mp = d.m + first;
     float* pp = d.p + first;
+    uint16_t* hp16 = d.p_bf16 ? d.p_bf16 + first : nullptr;
     const float* ap = d.ws_rowscale + q.row0 + q.ty;
-    const float ssr_k = d.scal[0] * d.scal[1];
+    const float ssr_k = d.scal[0] * d.scal[1] * hc.gscale;
     const float wd = (d.flags & kFlagNoWd) ? 0.f : hc.wd;
     const float nlr = -hc.lr, omb1 = hc.omb1;
     float b[VEC];
@@ -711,11 +743,13 @@ __device__ __forceinline__ void p34_adafactor_tile(const TensorDev& d, int rb, i
                 }
                 store_f<VEC>(mp + k * stride, mo[k]);
                 store_f<VEC>(pp + k * stride, th[k]);
+                if (hp16) store_bf16<VEC>(hp16 + k * stride, th[k]);
             }
         }
         gp += U * gstride;
         mp += U * stride;
         pp += U * stride;
+        if (hp16) hp16 += U * stride;
         ap += U * q.TY;
     }
 }
@@ -807,7 +841,7 @@ k_vec_second_moment(const TensorDev* __restrict__ T, const VChunk* __restrict__ 
     const long long i1 = min(d.rows, i0 + kVecChunk);
     float acc = 0.f;
     for (long long i = i0 + threadIdx.x; i < i1; i += kThreads) {
-        const float g = load_grad_scalar(d, i);
+        const float g = load_grad_scalar(d, i) * hc.gscale;
         const float vn = fmaf(hc.beta2, d.r[i], hc.omb2 * fmaf(g, g, hc.eps1));
         d.r[i] = vn;
         const float u = g * __frsqrt_rn(vn);
@@ -829,7 +863,7 @@ k_vec_apply(const TensorDev* __restrict__ T, const VChunk* __restrict__ chunks, 
     const float wd = (d.flags & kFlagNoWd) ? 0.f : hc.wd;
     const bool noconf = (d.flags & kFlagVecNoConf) != 0;
     for (long long i = i0 + threadIdx.x; i < i1; i += kThreads) {
-        const float g = load_grad_scalar(d, i);
+        const float g = load_grad_scalar(d, i) * hc.gscale;
         const float uh = (g * __frsqrt_rn(d.r[i])) * kappa;
         const float mo = d.m[i];
         const float e = uh - mo;
@@ -844,7 +878,9 @@ k_vec_apply(const TensorDev* __restrict__ T, const VChunk* __restrict__ chunks, 
             d.R[i] = Sn;
             dir = mn * __frsqrt_rn(Sn);
         }
-        d.p[i] = fmaf(-hc.lr, fmaf(wd, th, dir), th);
+        const float tn = fmaf(-hc.lr, fmaf(wd, th, dir), th);
+        d.p[i] = tn;
+        if (d.p_bf16) d.p_bf16[i] = static_cast<uint16_t>(pack_bf16x2(tn, 0.f) & 0xffffu);
     }
 }
 

@@ -59,7 +59,7 @@ def compare_state(opt, orc, indices=None) -> dict:
 
 def run_paired(torch, binding, oracle, w: synth.Workload, seed: int, steps: int, check_at,
                flags=None, hparams=None, device="cuda:0", oracle_idx=None, workers: int = 0,
-               algorithm: str = "came"):
+               algorithm: str = "came", bf16_copy: bool = False):
     """Step the CUDA path and the oracle side by side; returns {step: worst-error dict}.
 
     ``oracle_idx``: run the oracle on these tensors only (tensors are independent, so each is
@@ -70,7 +70,7 @@ def run_paired(torch, binding, oracle, w: synth.Workload, seed: int, steps: int,
     dev_p = [torch.from_numpy(p).to(device) for p in params]
     g0 = synth.make_grads(w, seed, 1, workers=workers)
     dev_g = [to_torch_grad(torch, g, device) for g in g0]
-    opt = binding.CameOptimizer(dev_p, dev_g, flags=flags,
+    opt = binding.CameOptimizer(dev_p, dev_g, flags=flags, bf16_copy=bf16_copy,
                                 create_flags=binding.CAME_CREATE_ADAFACTOR if algorithm == "adafactor" else 0)
     sel = list(range(len(params))) if oracle_idx is None else list(oracle_idx)
     no_wd = [bool(flags[i] & binding.CAME_T_NO_WEIGHT_DECAY) for i in sel] if flags else ()
@@ -85,10 +85,16 @@ def run_paired(torch, binding, oracle, w: synth.Workload, seed: int, steps: int,
             for dg, g in zip(dev_g, grads):
                 dg.copy_(to_torch_grad(torch, g, device))
         opt.step(**hp)
-        orc.step([synth.widen(grads[i]) for i in sel], **hp)
+        gs = float(hp.get("grad_scale", 1.0))       # the step's gradient is gs * buffer
+        orc.step([synth.widen(grads[i]) * gs for i in sel], **hp)
         g0 = None
         if step in check_at:
             torch.cuda.synchronize()
             out[step] = compare_state(opt, orc, None if oracle_idx is None else sel)
+            if bf16_copy:       # the copy is the kernel's own fp32 result rounded to nearest even
+                for p32, p16 in zip(opt.params, opt.p_bf16):
+                    want = synth.f32_to_bf16_bits(p32.cpu().numpy())
+                    got = p16.view(torch.int16).cpu().numpy().view(np.uint16)
+                    assert np.array_equal(got, want), "bf16 parameter copy is not RNE of the fp32 result"
     opt.close()
     return out

@@ -131,3 +131,30 @@ def test_adafactor_mode_needs_no_instability_state(env):
     assert err_signed(p[0].cpu().numpy(), orc.p[0]) <= TOL_STEP1
     assert err_signed(p[1].cpu().numpy(), orc.p[1]) <= TOL_STEP1
     binding.came_destroy(ctx)
+
+
+# ---------------------------------------------------------------------------
+# steps either side of the path, fused into its passes: gradient pre-scale, bf16 copy of theta
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("algorithm", ["came", "adafactor"])
+def test_grad_scale_and_bf16_copy(env, algorithm):
+    torch, binding, oracle = env
+    ts = (synth.mat("a", 257, 1032), synth.mat("b", 300, 516), synth.mat("c", 33, 65),
+          synth.vec("v", 1001))
+    for dt in (synth.BF16, synth.F32):
+        hp = dict(synth.PAPER_HPARAMS, grad_scale=1.0 / 48.0, eps1=1e-12)
+        w = synth.Workload("fused", ts, dt, "normal_fixed", 1e-3, 0.0, (), 10, hp)
+        _gate(run_paired(torch, binding, oracle, w, seed=23, steps=10, check_at=(1, 10),
+                         algorithm=algorithm, bf16_copy=True))
+
+
+def test_grad_scale_is_validated(env):
+    torch, binding, oracle = env
+    w = synth.workload("toy")
+    p = [torch.from_numpy(x).cuda() for x in synth.make_params(w, 1)]
+    g = [torch.from_numpy(x).cuda() for x in synth.make_grads(w, 1, 1)]
+    opt = binding.CameOptimizer(p, g)
+    with pytest.raises(binding.CameError) as e:
+        opt.step(**dict(w.hparams, grad_scale=-2.0))
+    assert e.value.status == 5
+    opt.close()
