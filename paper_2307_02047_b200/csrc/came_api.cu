@@ -30,6 +30,8 @@ long long g_tile_elems_override = 0;   // came_tune(CAME_TUNE_TILE_ELEMS)
 
 struct Plan {
     int vec = 1, tx = 256, tr = 0, n_rb = 0, n_cb = 0, n_seg = 0, n_parts = 0, kind = 0;
+    int n_grp = 0;
+    size_t counters() const { return static_cast<size_t>(n_rb) + n_cb + 2 + static_cast<size_t>(n_grp) * n_cb; }
 };
 
 inline long long ceil_div(long long a, long long b) { return (a + b - 1) / b; }
@@ -73,6 +75,7 @@ Plan plan_tensor(long long rows, long long cols, int ndim, int dtype, bool align
     p.n_rb = static_cast<int>(ceil_div(rows, tr));
     p.n_seg = p.n_cb * (p.tx / 32);
     p.n_parts = p.n_rb * p.n_cb;
+    p.n_grp = (p.n_rb + came::kColGroup - 1) / came::kColGroup;
     return p;
 }
 
@@ -370,7 +373,7 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
     std::vector<VChunk> chunks;
     size_t ws = 0;
     auto take = [&](size_t bytes) { const size_t off = ws; ws += (bytes + 255) / 256 * 256; return off; };
-    struct Off { size_t colpart, rowpart, blocksum, usq, cnt, scal, rowscale, colscale; };
+    struct Off { size_t colpart, colpart2, rowpart, blocksum, usq, cnt, scal, rowscale, colscale; };
     std::vector<Off> offs(n);
     for (int i = 0; i < n; ++i) {
         const came_tensor& x = t[i];
@@ -395,6 +398,7 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
             for (int rb = 0; rb < p.n_rb; ++rb)
                 for (int cb = 0; cb < p.n_cb; ++cb) tiles.push_back(Tile{i, rb, cb});
             offs[i].colpart = take(sizeof(float) * static_cast<size_t>(p.n_rb) * x.cols);
+            offs[i].colpart2 = take(sizeof(float) * static_cast<size_t>(p.n_grp) * x.cols);
             offs[i].rowpart = take(sizeof(float) * static_cast<size_t>(p.n_seg) * x.rows);
             offs[i].blocksum = take(sizeof(float) * p.n_rb);
             offs[i].rowscale = take(sizeof(float) * static_cast<size_t>(x.rows));
@@ -405,11 +409,11 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
             ctx->stream_bytes += numel * (sg + (conf ? 32 : 24));
             ctx->comp_bytes += numel * (sg + (conf ? 32 : 24));
             for (int c = 0; c < p.n_parts; ++c) chunks.push_back(VChunk{i, c});
-            offs[i].colpart = offs[i].rowpart = offs[i].blocksum = 0;
+            offs[i].colpart = offs[i].colpart2 = offs[i].rowpart = offs[i].blocksum = 0;
             offs[i].rowscale = offs[i].colscale = 0;
         }
         offs[i].usq = take(sizeof(float) * p.n_parts);
-        offs[i].cnt = take(sizeof(unsigned) * (p.n_rb + p.n_cb + 2));
+        offs[i].cnt = take(sizeof(unsigned) * p.counters());
         offs[i].scal = take(sizeof(float) * 4);
         if (tiles.size() > (1u << 30) || chunks.size() > (1u << 30)) {
             delete ctx;
@@ -452,6 +456,7 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
         d.p_bf16 = static_cast<uint16_t*>(x.param_bf16);
         d.rows = x.rows; d.cols = x.cols;
         d.ws_colpart = reinterpret_cast<float*>(ctx->d_ws + offs[i].colpart);
+        d.ws_colpart2 = reinterpret_cast<float*>(ctx->d_ws + offs[i].colpart2);
         d.ws_rowpart = reinterpret_cast<float*>(ctx->d_ws + offs[i].rowpart);
         d.ws_blocksum = reinterpret_cast<float*>(ctx->d_ws + offs[i].blocksum);
         d.ws_usq = reinterpret_cast<float*>(ctx->d_ws + offs[i].usq);
@@ -462,6 +467,7 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
         d.kind = p.kind; d.vec = p.vec;
         int lg = 0; while ((1 << lg) < p.tx) ++lg;
         d.tx_log2 = lg; d.tr = p.tr; d.n_rb = p.n_rb; d.n_cb = p.n_cb; d.n_seg = p.n_seg;
+        d.n_grp = p.n_grp;
         d.n_parts = p.n_parts; d.ndim = x.ndim; d.flags = x.flags;
         if (adafactor && x.ndim == 1) d.flags |= came::kFlagVecNoConf;   // Algorithm 1 has no S
         if (!(flags & CAME_CREATE_KEEP_STATE)) {
@@ -678,15 +684,16 @@ extern "C" came_status came_factor_update_static(const void* grad, int32_t grad_
     // Lay the scratch out; grow the tile until the partial sums fit (fewer, taller tiles).
     Plan p;
     size_t need = 0;
-    struct { size_t colpart, rowpart, blocksum, rowscale, colscale, cnt, scal; } off{};
+    struct { size_t colpart, colpart2, rowpart, blocksum, rowscale, colscale, cnt, scal; } off{};
     for (long long target = 32768; ; target *= 2) {
         p = plan_tensor(rows, cols, 2, grad_dtype, true, target);
         size_t ws = 0;
         auto take = [&](size_t bytes) { const size_t o = ws; ws += (bytes + 255) / 256 * 256; return o; };
-        off.cnt = take(sizeof(unsigned) * (static_cast<size_t>(p.n_rb) + p.n_cb + 2));
+        off.cnt = take(sizeof(unsigned) * p.counters());
         off.scal = take(sizeof(float) * 4);
         off.blocksum = take(sizeof(float) * p.n_rb);
         off.colpart = take(sizeof(float) * static_cast<size_t>(p.n_rb) * cols);
+        off.colpart2 = take(sizeof(float) * static_cast<size_t>(p.n_grp) * cols);
         off.rowpart = take(sizeof(float) * static_cast<size_t>(p.n_seg) * rows);
         off.rowscale = take(sizeof(float) * static_cast<size_t>(rows));
         off.colscale = take(sizeof(float) * static_cast<size_t>(cols));
@@ -728,6 +735,7 @@ extern "C" came_status came_factor_update_static(const void* grad, int32_t grad_
     d.scal = reinterpret_cast<float*>(base + off.scal);
     d.ws_blocksum = reinterpret_cast<float*>(base + off.blocksum);
     d.ws_colpart = reinterpret_cast<float*>(base + off.colpart);
+    d.ws_colpart2 = reinterpret_cast<float*>(base + off.colpart2);
     d.ws_rowpart = reinterpret_cast<float*>(base + off.rowpart);
     d.ws_rowscale = reinterpret_cast<float*>(base + off.rowscale);
     d.ws_colscale = reinterpret_cast<float*>(base + off.colscale);
@@ -735,6 +743,7 @@ extern "C" came_status came_factor_update_static(const void* grad, int32_t grad_
     d.kind = p.kind; d.vec = p.vec;
     int lg = 0; while ((1 << lg) < p.tx) ++lg;
     d.tx_log2 = lg; d.tr = p.tr; d.n_rb = p.n_rb; d.n_cb = p.n_cb; d.n_seg = p.n_seg;
+    d.n_grp = p.n_grp;
     d.n_parts = p.n_parts; d.ndim = 2; d.flags = 0;
 
     StepConsts hc;

@@ -13,9 +13,10 @@
 // rsqrt of every finished row and column factor is stored once by the tile that finishes it.
 //
 // Reductions are deterministic: every tile writes its partial sums to a
-// workspace and the LAST tile to arrive (per row block, per column strip, per
-// tensor; counted with atomics) adds them in a fixed order.  No thread ever
-// waits on another block, so there is no spin anywhere in this file.
+// workspace and the LAST tile to arrive (per row block; per group of 16 row
+// blocks of a column strip, then per strip; per tensor -- counted with atomics)
+// adds them in a fixed order.  No thread ever waits on another block, so there
+// is no spin anywhere in this file.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -44,6 +45,7 @@ namespace came {
 
 constexpr int kThreads = 256;
 constexpr int kVecChunk = 4096;       // vector elements per block in the vector kernels
+constexpr int kColGroup = 16;         // row blocks per group in the two-level column reduction
 
 enum Kind : int { kF32x4 = 0, kBF16x8 = 1, kF32x1 = 2, kBF16x1 = 3 };
 
@@ -57,12 +59,14 @@ struct TensorDev {
     float*       C;
     long long    rows, cols;
     float*       ws_colpart;   // [n_rb][cols]   per-tile column partial sums
+    float*       ws_colpart2;  // [n_grp][cols]  sums of kColGroup consecutive row blocks' partials
     float*       ws_rowpart;   // [n_seg][rows]  per-warp-segment row partial sums
     float*       ws_blocksum;  // [n_rb]         sum of the finished row factor over one row block
     float*       ws_usq;       // [n_parts]      per-tile partial sums of u^2
     float*       ws_rowscale;  // [rows]  rsqrt of the row factor last finished (r_t, then R_t)
     float*       ws_colscale;  // [cols]  rsqrt of the column factor last finished (c_t, then C_t)
-    unsigned*    cnt;          // [n_rb] row-block arrivals, [n_cb] strip arrivals, [1] finished, [1] usq
+    unsigned*    cnt;          // [n_rb] row-block arrivals, [n_cb] finished groups per strip,
+                               // [1] finished, [1] usq, [n_grp*n_cb] arrivals per (group, strip)
     float*       scal;         // [0] sqrt(sum r)  [1] kappa  [2] sqrt(sum R)
     uint16_t*    p_bf16;       // optional bf16 copy of the updated parameters (NULL = none)
     int          kind;
@@ -70,6 +74,7 @@ struct TensorDev {
     int          tx_log2;      // threads across columns = 1 << tx_log2 (32..256)
     int          tr;           // rows per tile
     int          n_rb, n_cb, n_seg;
+    int          n_grp;        // ceil(n_rb / kColGroup)
     int          n_parts;      // matrices: n_rb*n_cb; vectors: number of chunks
     int          ndim;
     unsigned     flags;
@@ -226,6 +231,41 @@ template <> struct Log2<2> { static constexpr int v = 1; };
 template <> struct Log2<4> { static constexpr int v = 2; };
 template <> struct Log2<8> { static constexpr int v = 3; };
 
+// Adds `count` (<= kColGroup) rows of partial sums, `stride` floats apart, for VW adjacent
+// columns: eight rows are fetched per round trip to L2 before they are added, and the adds
+// run in row order, so the result does not depend on timing.
+template <int VW>
+__device__ __forceinline__ void sum_partial_rows(const float* __restrict__ p, long long stride,
+                                                 int count, float (&acc)[VW])
+{
+    constexpr int B = 8;                       // rows fetched per round trip
+#pragma unroll
+    for (int j = 0; j < VW; ++j) acc[j] = 0.f;
+#pragma unroll
+    for (int k0 = 0; k0 < kColGroup; k0 += B) {
+        if (k0 >= count) break;
+        float v[B][VW];
+#pragma unroll
+        for (int k = 0; k < B; ++k) {
+            if (k0 + k < count) {
+                if constexpr (VW == 4) {
+                    const float4 t = __ldcg(reinterpret_cast<const float4*>(p + (k0 + k) * stride));
+                    v[k][0] = t.x; v[k][1] = t.y; v[k][2] = t.z; v[k][3] = t.w;
+                } else {
+                    v[k][0] = __ldcg(p + (k0 + k) * stride);
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < VW; ++j) v[k][j] = 0.f;
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < B; ++k)
+#pragma unroll
+            for (int j = 0; j < VW; ++j) acc[j] += v[k][j];
+    }
+}
+
 // ---------------------------------------------------------------------------
 // Last-arriver finalisation of one factored EMA (Algorithm 2: r_t, c_t from g^2
 // with beta2/eps1; R_t, C_t from U_t with beta3/eps2):
@@ -241,18 +281,21 @@ __device__ __forceinline__ void finalize_factors(const TensorDev& d, int rb, int
                                                  float* __restrict__ colfac,
                                                  float* __restrict__ sqrt_sum, Shared& sm)
 {
-    const int tid = threadIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int grp = rb / kColGroup;
+    const int grp_size = min(kColGroup, d.n_rb - grp * kColGroup);
+    unsigned* const cnt_grp = d.cnt + d.n_rb + d.n_cb + 2;
     __threadfence();
     __syncthreads();
     if (tid == 0) {
         const unsigned a = atomicAdd(&d.cnt[rb], 1u);
-        const unsigned b = atomicAdd(&d.cnt[d.n_rb + cb], 1u);
+        const unsigned b = atomicAdd(&cnt_grp[grp * d.n_cb + cb], 1u);
         sm.flag[0] = (a == static_cast<unsigned>(d.n_cb - 1));
-        sm.flag[1] = (b == static_cast<unsigned>(d.n_rb - 1));
+        sm.flag[1] = (b == static_cast<unsigned>(grp_size - 1));
     }
     __syncthreads();
-    const bool last_r = sm.flag[0] != 0, last_c = sm.flag[1] != 0;
-    if (!last_r && !last_c) return;
+    const bool last_r = sm.flag[0] != 0, last_g = sm.flag[1] != 0;
+    if (!last_r && !last_g) return;
     __threadfence();
 
     const long long rows = d.rows, cols = d.cols;
@@ -261,41 +304,95 @@ __device__ __forceinline__ void finalize_factors(const TensorDev& d, int rb, int
         const long long row1 = min(rows, row0 + d.tr);
         const float add = static_cast<float>(cols) * eps;
         float bs = 0.f;
-        for (long long row = row0 + tid; row < row1; row += kThreads) {
-            float s = 0.f;
-            for (int sg = 0; sg < d.n_seg; ++sg) s += __ldcg(d.ws_rowpart + sg * rows + row);
-            const float nv = fmaf(beta, rowfac[row], omb * fmaf(scale, s, add));
-            rowfac[row] = nv;
-            d.ws_rowscale[row] = __frsqrt_rn(nv);
-            bs += nv;
+        if (d.n_seg <= 32) {
+            // few segments per row: one thread per row, segments added in order
+            for (long long row = row0 + tid; row < row1; row += kThreads) {
+                float s = 0.f;
+#pragma unroll 8
+                for (int sg = 0; sg < d.n_seg; ++sg) s += __ldcg(d.ws_rowpart + sg * rows + row);
+                const float nv = fmaf(beta, rowfac[row], omb * fmaf(scale, s, add));
+                rowfac[row] = nv;
+                d.ws_rowscale[row] = __frsqrt_rn(nv);
+                bs += nv;
+            }
+        } else {
+            // many segments: one warp per row, lanes stride over the segments, fixed shuffle tree
+            for (long long row = row0 + warp; row < row1; row += kThreads / 32) {
+                float s = 0.f;
+#pragma unroll 4
+                for (int sg = lane; sg < d.n_seg; sg += 32) s += __ldcg(d.ws_rowpart + sg * rows + row);
+                s = warp_sum(s);
+                if (lane == 0) {
+                    const float nv = fmaf(beta, rowfac[row], omb * fmaf(scale, s, add));
+                    rowfac[row] = nv;
+                    d.ws_rowscale[row] = __frsqrt_rn(nv);
+                    bs += nv;
+                }
+            }
         }
-        bs = block_sum(bs, sm);
+        bs = block_sum(bs, sm);          // fixed order: warp tree, then warps 0..7
         if (tid == 0) { d.ws_blocksum[rb] = bs; d.cnt[rb] = 0u; }
     }
-    if (last_c) {
+    bool last_c = false;
+    if (last_g) {
+        // level 1: this group's (<= kColGroup) row-block partials of the strip -> one group partial
         const int sw = (1 << d.tx_log2) * d.vec;
         const long long col0 = static_cast<long long>(cb) * sw;
         const long long col1 = min(cols, col0 + sw);
-        const float add = static_cast<float>(rows) * eps;
-        for (long long col = col0 + tid; col < col1; col += kThreads) {
-            float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-            const float* pc = d.ws_colpart + col;
-            int k = 0;
-            for (; k + 4 <= d.n_rb; k += 4) {      // fixed association, see the sum below
-                s0 += __ldcg(pc + (k + 0) * cols);
-                s1 += __ldcg(pc + (k + 1) * cols);
-                s2 += __ldcg(pc + (k + 2) * cols);
-                s3 += __ldcg(pc + (k + 3) * cols);
+        const int rb0 = grp * kColGroup;
+        const float* src = d.ws_colpart + static_cast<long long>(rb0) * cols;
+        float* dst = d.ws_colpart2 + static_cast<long long>(grp) * cols;
+        if (d.vec >= 4) {
+            for (long long col = col0 + 4 * tid; col < col1; col += 4 * kThreads) {
+                float acc[4];
+                sum_partial_rows<4>(src + col, cols, grp_size, acc);
+                *reinterpret_cast<float4*>(dst + col) = make_float4(acc[0], acc[1], acc[2], acc[3]);
             }
-            for (; k < d.n_rb; ++k) s0 += __ldcg(pc + k * cols);
-            const float s = (s0 + s1) + (s2 + s3);
-            const float nv = fmaf(beta, colfac[col], omb * fmaf(scale, s, add));
-            colfac[col] = nv;
-            d.ws_colscale[col] = __frsqrt_rn(nv);
+        } else {
+            for (long long col = col0 + tid; col < col1; col += kThreads) {
+                float acc[1];
+                sum_partial_rows<1>(src + col, cols, grp_size, acc);
+                dst[col] = acc[0];
+            }
         }
-        if (tid == 0) d.cnt[d.n_rb + cb] = 0u;
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) {
+            cnt_grp[grp * d.n_cb + cb] = 0u;
+            const unsigned c = atomicAdd(&d.cnt[d.n_rb + cb], 1u);
+            sm.flag[1] = (c == static_cast<unsigned>(d.n_grp - 1));
+        }
+        __syncthreads();
+        last_c = sm.flag[1] != 0;
+        if (last_c) {
+            // level 2: the strip's group partials -> EMA, factor and its rsqrt
+            __threadfence();
+            const float add = static_cast<float>(rows) * eps;
+            if (d.vec >= 4) {
+                for (long long col = col0 + 4 * tid; col < col1; col += 4 * kThreads) {
+                    float acc[4];
+                    sum_partial_rows<4>(d.ws_colpart2 + col, cols, d.n_grp, acc);
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        const float nv = fmaf(beta, colfac[col + j], omb * fmaf(scale, acc[j], add));
+                        colfac[col + j] = nv;
+                        d.ws_colscale[col + j] = __frsqrt_rn(nv);
+                    }
+                }
+            } else {
+                for (long long col = col0 + tid; col < col1; col += kThreads) {
+                    float acc[1];
+                    sum_partial_rows<1>(d.ws_colpart2 + col, cols, d.n_grp, acc);
+                    const float nv = fmaf(beta, colfac[col], omb * fmaf(scale, acc[0], add));
+                    colfac[col] = nv;
+                    d.ws_colscale[col] = __frsqrt_rn(nv);
+                }
+            }
+            if (tid == 0) d.cnt[d.n_rb + cb] = 0u;
+        }
     }
     const unsigned done = (last_r ? 1u : 0u) + (last_c ? 1u : 0u);
+    if (done == 0u) return;
     __threadfence();
     __syncthreads();
     if (tid == 0) {
