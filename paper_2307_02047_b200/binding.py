@@ -206,7 +206,10 @@ def make_hparams(step: int, **kw) -> came_hparams:
 class CameOptimizer:
     """Owns the CAME state for a list of torch CUDA parameter tensors and steps them.
 
-    ``params``: fp32 CUDA tensors (1-D or 2-D, contiguous), updated in place.
+    ``params``: fp32 CUDA tensors (contiguous), updated in place.  1-D tensors take the vector
+    path, 2-D tensors the matrix path; a tensor of rank >= 3 is handed to the library as the
+    matrix (product of the leading dims) x (last dim), since the paper defines the method for
+    matrices only.
     ``grads``: CUDA tensors of the same shapes, fp32 or bf16, read every step
     (their storage may be refilled between steps; pointers are fixed at creation).
     torch is used for allocation and the stream only.
@@ -223,20 +226,21 @@ class CameOptimizer:
         for i, (p, g) in enumerate(zip(self.params, self.grads)):
             assert p.is_cuda and p.dtype == torch.float32 and p.is_contiguous()
             assert g.is_cuda and g.is_contiguous() and g.shape == p.shape
-            assert p.dim() in (1, 2)
-            rows = p.shape[0]
-            cols = p.shape[1] if p.dim() == 2 else 1
+            assert p.dim() >= 1
+            ndim = 1 if p.dim() == 1 else 2
+            cols = p.shape[-1] if ndim == 2 else 1
+            rows = p.numel() // cols
             z = lambda n: torch.empty(n, dtype=torch.float32, device=p.device)
             self.m.append(torch.empty_like(p))
             self.r.append(z(rows)); self.R.append(z(rows))
-            self.c.append(z(cols) if p.dim() == 2 else None)
-            self.C.append(z(cols) if p.dim() == 2 else None)
+            self.c.append(z(cols) if ndim == 2 else None)
+            self.C.append(z(cols) if ndim == 2 else None)
             gd = CAME_BF16 if g.dtype == torch.bfloat16 else CAME_F32
             assert g.dtype in (torch.bfloat16, torch.float32)
             ptr = lambda t: t.data_ptr() if t is not None else None
             self.p_bf16.append(torch.empty_like(p, dtype=torch.bfloat16) if bf16_copy else None)
             descs.append(came_tensor(ptr(p), ptr(g), ptr(self.m[i]), ptr(self.r[i]), ptr(self.c[i]),
-                                     ptr(self.R[i]), ptr(self.C[i]), rows, cols, p.dim(), gd,
+                                     ptr(self.R[i]), ptr(self.C[i]), rows, cols, ndim, gd,
                                      0 if flags is None else int(flags[i]), 0, ptr(self.p_bf16[i])))
         self.ctx = came_create(descs, device=device, flags=create_flags)
         self.step_count = 0

@@ -209,3 +209,53 @@ def test_queries_and_profiling(env):
                      "p4_apply", "vec_apply"]
     assert all(0.0 < x < 50.0 for x in ms)
     binding.came_destroy(ctx)
+
+
+def test_rank3_tensor_is_the_matrix_of_merged_leading_dims(env, oracle):
+    torch, binding = env
+    from tests.parity_util import err_signed
+    w = synth.workload("mat:96x520")
+    p0 = synth.make_params(w, 31)[0]
+    g0 = synth.make_grad(w, 31, 0, 1)
+    p = torch.from_numpy(p0.reshape(8, 12, 520).copy()).cuda()
+    g = torch.from_numpy(g0.reshape(8, 12, 520).copy()).cuda()
+    opt = binding.CameOptimizer([p], [g])
+    opt.step(**HP)
+    torch.cuda.synchronize()
+    orc = oracle.OracleOptimizer([p0])
+    orc.step([synth.widen(g0)], **HP)
+    assert p.shape == (8, 12, 520)
+    assert err_signed(p.cpu().numpy().reshape(96, 520), orc.p[0]) <= 1e-5
+    opt.close()
+
+
+def test_cuda_graph_replay_matches_eager_launches(env):
+    """came_step neither synchronises nor allocates, so a caller may capture it in a CUDA graph
+    and replay it; the replayed steps must equal eagerly launched ones bit for bit."""
+    torch, binding = env
+    a = Buffers(torch, binding, W_ODD, 13)
+    ctx = binding.came_create(a.descs)
+    a.set_grads(13, 1)
+    for step in (1, 2, 3, 4):
+        binding.came_step(ctx, binding.make_hparams(step, **HP), None, torch.cuda.current_stream().cuda_stream)
+    torch.cuda.synchronize()
+    binding.came_destroy(ctx)
+
+    b = Buffers(torch, binding, W_ODD, 13)
+    ctx = binding.came_create(b.descs)
+    b.set_grads(13, 1)
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        binding.came_step(ctx, binding.make_hparams(1, **HP), None, side.cuda_stream)   # warm-up, eager
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        binding.came_step(ctx, binding.make_hparams(2, **HP), None,
+                          torch.cuda.current_stream().cuda_stream)
+    for _ in range(3):          # steps 2, 3, 4 (capture itself runs nothing)
+        graph.replay()
+    torch.cuda.synchronize()
+    binding.came_destroy(ctx)
+    assert _same(a.snapshot(), b.snapshot())

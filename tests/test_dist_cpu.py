@@ -54,3 +54,82 @@ def test_reference_arm_other_ranks_do_nothing():
                           "--steps", "1", "--warmup", "0"], env=env, capture_output=True,
                          text=True, timeout=120)
     assert res.returncode == 0 and res.stdout.strip() == ""
+
+
+# ---------------------------------------------------------------------------
+# tensor-sharded step: two gloo ranks, the oracle as the injected local stepper
+# ---------------------------------------------------------------------------
+def test_partition_by_bytes_balances_and_is_deterministic():
+    sys.path.insert(0, ROOT)
+    from paper_2307_02047_b200.sharded import partition_by_bytes
+    sizes = [100, 90, 50, 40, 30, 10, 10, 5]
+    own = partition_by_bytes(sizes, 2)
+    loads = [sum(s for s, o in zip(sizes, own) if o == r) for r in range(2)]
+    assert abs(loads[0] - loads[1]) <= max(sizes) and sum(loads) == sum(sizes)
+    assert own == partition_by_bytes(sizes, 2)
+    assert partition_by_bytes(sizes, 1) == [0] * len(sizes)
+    assert sorted(set(partition_by_bytes([7] * 8, 8))) == list(range(8))
+
+
+def _sharded_worker(rank, world, port, q):
+    sys.path.insert(0, ROOT)
+    import numpy as np
+    from oracle import came_oracle
+    from paper_2307_02047_b200 import synth
+    from paper_2307_02047_b200.sharded import ShardedCame
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    ts = (synth.mat("a", 24, 40), synth.mat("b", 16, 8), synth.vec("v", 33), synth.mat("c", 5, 64))
+    hp = dict(synth.PAPER_HPARAMS, weight_decay=0.01)
+    w = synth.Workload("sh", ts, synth.F32, "normal_fixed", 1e-3, 0.0, (), 3, hp)
+    params = [torch.from_numpy(x.astype(np.float64)) for x in synth.make_params(w, 1)]
+    grads = [torch.zeros_like(p) for p in params]
+
+    class OracleLocal:                      # stands in for the CUDA context on this CPU test
+        def __init__(self, p, g):
+            self.p, self.g = p, g
+            self.o = came_oracle.OracleOptimizer([x.numpy() for x in p])
+        def step(self, **h):
+            gs = h.pop("grad_scale")
+            self.o.step([x.numpy() * gs for x in self.g], **h)
+            for dst, src in zip(self.p, self.o.p):
+                dst.copy_(torch.from_numpy(src))
+
+    sh = ShardedCame(params, grads, make_local=OracleLocal)
+    for step in (1, 2, 3):
+        for i, g in enumerate(grads):       # each rank has its own micro-batch gradient
+            g.copy_(torch.from_numpy(synth.widen(synth.make_grad(w, 100 + rank, i, step))))
+        sh.step(**hp)
+    q.put((rank, sh.owner, [p.numpy().copy() for p in params]))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_sharded_step_equals_single_process_mean_gradient():
+    import numpy as np
+    sys.path.insert(0, ROOT)
+    from oracle import came_oracle
+    from paper_2307_02047_b200 import synth
+    ctx = mp.get_context("spawn")
+    q = ctx.Queue()
+    port = 31500 + os.getpid() % 2000
+    procs = [ctx.Process(target=_sharded_worker, args=(r, 2, port, q)) for r in range(2)]
+    for p in procs:
+        p.start()
+    out = sorted((q.get(timeout=180) for _ in procs), key=lambda o: o[0])
+    for p in procs:
+        p.join(timeout=60)
+        assert p.exitcode == 0
+    assert out[0][1] == out[1][1] and set(out[0][1]) == {0, 1}       # same partition, both ranks used
+    # reference: one process stepping on the mean of the two ranks' gradients
+    ts = (synth.mat("a", 24, 40), synth.mat("b", 16, 8), synth.vec("v", 33), synth.mat("c", 5, 64))
+    hp = dict(synth.PAPER_HPARAMS, weight_decay=0.01)
+    w = synth.Workload("sh", ts, synth.F32, "normal_fixed", 1e-3, 0.0, (), 3, hp)
+    ref = came_oracle.OracleOptimizer(synth.make_params(w, 1))
+    for step in (1, 2, 3):
+        gs = [(synth.widen(synth.make_grad(w, 100, i, step)) + synth.widen(synth.make_grad(w, 101, i, step))) * 0.5
+              for i in range(len(ts))]
+        ref.step(gs, **hp)
+    for r in range(2):
+        for got, want in zip(out[r][2], ref.p):
+            np.testing.assert_allclose(got, want, rtol=1e-12, atol=0)
