@@ -166,7 +166,11 @@ came_status came_step(came_ctx* ctx, const came_hparams* hp, const void* const* 
  * host_grads[i] (HOST, grad_dtype [rows*cols], ideally pinned) into the tensor's
  * device gradient buffer, runs the step, then, where host_params_out is not NULL
  * and host_params_out[i] is not NULL, copies the updated parameters back (HOST,
- * fp32 [rows*cols]).  All on `cuda_stream`, asynchronous for pinned memory. */
+ * fp32 [rows*cols]).  Tensors are independent in Algorithm 2, so the work is
+ * pipelined over groups of consecutive tensors on two internal copy streams:
+ * uploads, the step and downloads of different groups overlap.  Everything is
+ * ordered after the work already on `cuda_stream`, and `cuda_stream` waits for the
+ * last download, so synchronising it is enough.  Asynchronous for pinned memory. */
 came_status came_step_host(came_ctx* ctx, const came_hparams* hp, const void* const* host_grads,
                            void* const* host_params_out, void* cuda_stream);
 
@@ -235,11 +239,19 @@ came_status came_factor_update_static(const void* grad, int32_t grad_dtype, int6
                                       double eps1, float* out_sqrt_sum_r, int32_t device,
                                       void* cuda_stream);
 
-/* Process-wide tuning knob, read by later came_create calls.  CAME_TUNE_TILE_ELEMS:
+/* Process-wide tuning knobs, read by later came_create calls.  CAME_TUNE_TILE_ELEMS:
  * elements per matrix tile (0 restores the default, which scales with the size
- * of the parameter set).  Changes scheduling only, never results beyond the
+ * of the parameter set).  They change scheduling only, never results beyond the
  * order of the partial sums. */
-enum { CAME_TUNE_TILE_ELEMS = 0 };
+enum {
+    CAME_TUNE_TILE_ELEMS = 0,
+    CAME_TUNE_SCHED_GROUP_BYTES = 1,  /* > 0: came_step runs all phases of one group of consecutive
+                                         tensors (about this many bytes of g, m and theta) before
+                                         the next group, instead of one grid per phase over all
+                                         tensors; per-phase timing is then not reported.  0 = off. */
+    CAME_TUNE_HOST_GROUP_BYTES = 2    /* bytes of gradients + parameters per pipeline stage of
+                                         came_step_host (default 1 GiB) */
+};
 came_status came_tune(int32_t key, int64_t value);
 
 #ifdef __cplusplus

@@ -25,6 +25,8 @@ CAME_CREATE_ADAFACTOR = 2
  CAME_Q_WORKSPACE_BYTES, CAME_Q_NUM_TILES, CAME_Q_LAUNCHES_PER_STEP, CAME_Q_LAST_STEP,
  CAME_Q_NUM_PHASES, CAME_Q_MATRIX_NUMEL) = range(10)
 CAME_TUNE_TILE_ELEMS = 0
+CAME_TUNE_SCHED_GROUP_BYTES = 1
+CAME_TUNE_HOST_GROUP_BYTES = 2
 
 EXPORTED = ["came_create", "came_step", "came_step_host", "came_destroy", "came_last_error",
             "came_status_string", "came_query", "came_set_profiling", "came_get_phase_ms",

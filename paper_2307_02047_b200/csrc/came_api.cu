@@ -27,6 +27,8 @@ const char* const kPhaseNames[kMaxPhases] = {
 
 thread_local std::string g_create_error;
 long long g_tile_elems_override = 0;   // came_tune(CAME_TUNE_TILE_ELEMS)
+long long g_sched_group_bytes = 0;     // came_tune(CAME_TUNE_SCHED_GROUP_BYTES); 0 = one group
+long long g_host_group_bytes = 1ll << 30;   // came_tune(CAME_TUNE_HOST_GROUP_BYTES)
 
 struct Plan {
     int vec = 1, tx = 256, tr = 0, n_rb = 0, n_cb = 0, n_seg = 0, n_parts = 0, kind = 0;
@@ -81,6 +83,9 @@ Plan plan_tensor(long long rows, long long cols, int ndim, int dtype, bool align
 
 }  // namespace
 
+// A run of consecutive tensors handled together: [t0, t1) with their tiles and vector chunks.
+struct Group { int t0, t1, tile0, tile1, chunk0, chunk1; };
+
 struct came_ctx {
     int device = 0;
     int n = 0;
@@ -94,6 +99,12 @@ struct came_ctx {
     Tile* d_tiles = nullptr;
     VChunk* d_chunks = nullptr;
     int n_tiles = 0, n_chunks = 0;
+    std::vector<int> tile_begin, chunk_begin;   // [n+1] first tile / vector chunk of each tensor
+    std::vector<Group> sched_groups;            // device-resident step: launch order (empty = one grid)
+    std::vector<Group> host_groups;             // host-buffer step: pipeline stages
+    cudaStream_t s_up = nullptr, s_down = nullptr;   // copy streams of the host-buffer step
+    std::vector<cudaEvent_t> ev_up, ev_done;         // per host group: gradients landed / step done
+    cudaEvent_t ev_start = nullptr, ev_all_down = nullptr;
     char* d_ws = nullptr;
     size_t ws_bytes = 0, table_bytes = 0;
     long long numel = 0, matrix_numel = 0, state_bytes = 0, stream_bytes = 0, comp_bytes = 0;
@@ -209,6 +220,12 @@ void free_ctx(came_ctx* ctx)
     }
     for (cudaEvent_t e : ctx->prof_ev)
         if (e) cudaEventDestroy(e);
+    for (cudaEvent_t e : ctx->ev_up) if (e) cudaEventDestroy(e);
+    for (cudaEvent_t e : ctx->ev_done) if (e) cudaEventDestroy(e);
+    if (ctx->ev_start) cudaEventDestroy(ctx->ev_start);
+    if (ctx->ev_all_down) cudaEventDestroy(ctx->ev_all_down);
+    if (ctx->s_up) cudaStreamDestroy(ctx->s_up);
+    if (ctx->s_down) cudaStreamDestroy(ctx->s_down);
     delete ctx;
 }
 
@@ -232,50 +249,81 @@ came_status upload_table(came_ctx* ctx, cudaStream_t stream)
     return CAME_OK;
 }
 
-came_status launch_step(came_ctx* ctx, const came_hparams* hp, cudaStream_t stream)
+// Enqueue the kernels of one step for the tensors of `g` (all phases, in dependency order).
+// `ev` (may be NULL) receives one event before the first kernel and one after each kernel.
+int launch_range(const came_ctx* ctx, const StepConsts& hc, cudaStream_t stream, const Group& g,
+                 cudaEvent_t* ev)
 {
-    const StepConsts hc = make_consts(*hp);
-    const bool prof = ctx->profiling && !ctx->prof_ev.empty();
     int iv = 0;
-    cudaEvent_t* ev = prof ? &ctx->prof_ev[(ctx->prof_count % kProfSlots) * (kMaxPhases + 1)] : nullptr;
-    auto mark = [&](int slot) { if (prof) cudaEventRecord(ev[slot], stream); };
+    auto mark = [&](int slot) { if (ev) cudaEventRecord(ev[slot], stream); };
+    const int nt = g.tile1 - g.tile0, nc = g.chunk1 - g.chunk0;
+    const Tile* tiles = ctx->d_tiles + g.tile0;
+    const VChunk* chunks = ctx->d_chunks + g.chunk0;
     mark(0);
-    if (ctx->n_chunks > 0) {
-        came::k_vec_second_moment<<<ctx->n_chunks, came::kThreads, 0, stream>>>(
-            ctx->d_table, ctx->d_chunks, hc);
+    if (nc > 0) {
+        came::k_vec_second_moment<<<nc, came::kThreads, 0, stream>>>(ctx->d_table, chunks, hc);
         mark(++iv);
     }
-    if (ctx->n_tiles > 0) {
-        came::k_p1_reduce_g2<<<ctx->n_tiles, came::kThreads, 0, stream>>>(
-            ctx->d_table, ctx->d_tiles, ctx->n_tiles, 0, hc);
+    if (nt > 0) {
+        came::k_p1_reduce_g2<<<nt, came::kThreads, 0, stream>>>(ctx->d_table, tiles, nt, 0, hc);
         mark(++iv);
-        came::k_p2_sum_u2<<<ctx->n_tiles, came::kThreads, 0, stream>>>(
-            ctx->d_table, ctx->d_tiles, ctx->n_tiles, 1, hc);
+        came::k_p2_sum_u2<<<nt, came::kThreads, 0, stream>>>(ctx->d_table, tiles, nt, 1, hc);
         mark(++iv);
         if (ctx->adafactor) {
-            came::k_p34_adafactor_apply<<<ctx->n_tiles, came::kThreads, 0, stream>>>(
-                ctx->d_table, ctx->d_tiles, ctx->n_tiles, 0, hc);
+            came::k_p34_adafactor_apply<<<nt, came::kThreads, 0, stream>>>(ctx->d_table, tiles, nt, 0, hc);
             mark(++iv);
         } else {
-            came::k_p3_momentum_instability<<<ctx->n_tiles, came::kThreads, 0, stream>>>(
-                ctx->d_table, ctx->d_tiles, ctx->n_tiles, 0, hc);
+            came::k_p3_momentum_instability<<<nt, came::kThreads, 0, stream>>>(ctx->d_table, tiles, nt, 0, hc);
             mark(++iv);
-            came::k_p4_apply<<<ctx->n_tiles, came::kThreads, 0, stream>>>(
-                ctx->d_table, ctx->d_tiles, ctx->n_tiles, 1, hc);
+            came::k_p4_apply<<<nt, came::kThreads, 0, stream>>>(ctx->d_table, tiles, nt, 1, hc);
             mark(++iv);
         }
     }
-    if (ctx->n_chunks > 0) {
-        came::k_vec_apply<<<ctx->n_chunks, came::kThreads, 0, stream>>>(
-            ctx->d_table, ctx->d_chunks, hc);
+    if (nc > 0) {
+        came::k_vec_apply<<<nc, came::kThreads, 0, stream>>>(ctx->d_table, chunks, hc);
         mark(++iv);
     }
-    ctx->n_intervals = iv;
-    if (prof) ++ctx->prof_count;
+    return iv;
+}
+
+came_status launch_step(came_ctx* ctx, const came_hparams* hp, cudaStream_t stream)
+{
+    const StepConsts hc = make_consts(*hp);
+    if (ctx->sched_groups.empty()) {
+        const bool prof = ctx->profiling && !ctx->prof_ev.empty();
+        cudaEvent_t* ev = prof ? &ctx->prof_ev[(ctx->prof_count % kProfSlots) * (kMaxPhases + 1)] : nullptr;
+        const Group all{0, ctx->n, 0, ctx->n_tiles, 0, ctx->n_chunks};
+        ctx->n_intervals = launch_range(ctx, hc, stream, all, ev);
+        if (prof) ++ctx->prof_count;
+    } else {
+        // grouped schedule: all phases of one group before the next group starts, so that a
+        // group sized to the L2 re-reads its gradients and momentum from there
+        for (const Group& g : ctx->sched_groups) launch_range(ctx, hc, stream, g, nullptr);
+        ctx->n_intervals = 0;
+    }
     const cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(ctx, e, "kernel launch");
     ctx->last_step = hp->step;
     return CAME_OK;
+}
+
+// Consecutive tensors are grouped until a group holds `limit` bytes (by `bytes_of`).
+template <typename F>
+std::vector<Group> make_groups(const came_ctx* ctx, long long limit, F bytes_of)
+{
+    std::vector<Group> out;
+    int t0 = 0;
+    long long acc = 0;
+    for (int i = 0; i < ctx->n; ++i) {
+        acc += bytes_of(ctx->tensors[i]);
+        if (acc >= limit || i == ctx->n - 1) {
+            out.push_back(Group{t0, i + 1, ctx->tile_begin[t0], ctx->tile_begin[i + 1],
+                                ctx->chunk_begin[t0], ctx->chunk_begin[i + 1]});
+            t0 = i + 1;
+            acc = 0;
+        }
+    }
+    return out;
 }
 
 }  // namespace
@@ -308,8 +356,13 @@ const char* came_last_error(const came_ctx* ctx)
 
 came_status came_tune(int32_t key, int64_t value)
 {
-    if (key != CAME_TUNE_TILE_ELEMS || value < 0) return CAME_ERR_UNSUPPORTED;
-    g_tile_elems_override = value;
+    if (value < 0) return CAME_ERR_UNSUPPORTED;
+    switch (key) {
+        case CAME_TUNE_TILE_ELEMS: g_tile_elems_override = value; break;
+        case CAME_TUNE_SCHED_GROUP_BYTES: g_sched_group_bytes = value; break;
+        case CAME_TUNE_HOST_GROUP_BYTES: g_host_group_bytes = value > 0 ? value : (1ll << 30); break;
+        default: return CAME_ERR_UNSUPPORTED;
+    }
     return CAME_OK;
 }
 
@@ -369,6 +422,8 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
         while (target < 262144 && target * 2 * 2400 <= matrix_numel) target *= 2;
     }
     std::vector<Plan> plans(n);
+    ctx->tile_begin.assign(n + 1, 0);
+    ctx->chunk_begin.assign(n + 1, 0);
     std::vector<Tile> tiles;
     std::vector<VChunk> chunks;
     size_t ws = 0;
@@ -415,6 +470,8 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
         offs[i].usq = take(sizeof(float) * p.n_parts);
         offs[i].cnt = take(sizeof(unsigned) * p.counters());
         offs[i].scal = take(sizeof(float) * 4);
+        ctx->tile_begin[i + 1] = static_cast<int>(tiles.size());
+        ctx->chunk_begin[i + 1] = static_cast<int>(chunks.size());
         if (tiles.size() > (1u << 30) || chunks.size() > (1u << 30)) {
             delete ctx;
             return fail(nullptr, CAME_ERR_SHAPE, "too many tiles");
@@ -447,6 +504,24 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
         CAME_TRY(cudaEventCreateWithFlags(&ctx->pinned_free[k], cudaEventDisableTiming), "cudaEventCreate");
     }
 
+    {
+        auto state_bytes = [](const came_tensor& x) {
+            return x.rows * x.cols * (8ll + (x.grad_dtype == CAME_BF16 ? 2 : 4)); };
+        auto xfer_bytes = [](const came_tensor& x) {
+            return x.rows * x.cols * (4ll + (x.grad_dtype == CAME_BF16 ? 2 : 4)); };
+        if (g_sched_group_bytes > 0) ctx->sched_groups = make_groups(ctx, g_sched_group_bytes, state_bytes);
+        ctx->host_groups = make_groups(ctx, g_host_group_bytes, xfer_bytes);
+        CAME_TRY(cudaStreamCreateWithFlags(&ctx->s_up, cudaStreamNonBlocking), "cudaStreamCreate");
+        CAME_TRY(cudaStreamCreateWithFlags(&ctx->s_down, cudaStreamNonBlocking), "cudaStreamCreate");
+        CAME_TRY(cudaEventCreateWithFlags(&ctx->ev_start, cudaEventDisableTiming), "cudaEventCreate");
+        CAME_TRY(cudaEventCreateWithFlags(&ctx->ev_all_down, cudaEventDisableTiming), "cudaEventCreate");
+        ctx->ev_up.assign(ctx->host_groups.size(), nullptr);
+        ctx->ev_done.assign(ctx->host_groups.size(), nullptr);
+        for (cudaEvent_t& ev : ctx->ev_up)
+            CAME_TRY(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming), "cudaEventCreate");
+        for (cudaEvent_t& ev : ctx->ev_done)
+            CAME_TRY(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming), "cudaEventCreate");
+    }
     for (int i = 0; i < n; ++i) {
         const came_tensor& x = t[i];
         const Plan& p = plans[i];
@@ -525,25 +600,49 @@ came_status came_step_host(came_ctx* ctx, const came_hparams* hp, const void* co
     for (int i = 0; i < ctx->n; ++i)
         if (!host_grads[i]) return fail(ctx, CAME_ERR_NULL, "a host gradient pointer is NULL");
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-    for (int i = 0; i < ctx->n; ++i) {
-        const came_tensor& x = ctx->tensors[i];
-        const size_t bytes = static_cast<size_t>(x.rows) * x.cols * (x.grad_dtype == CAME_BF16 ? 2 : 4);
-        const cudaError_t e = cudaMemcpyAsync(const_cast<void*>(x.grad), host_grads[i], bytes,
-                                              cudaMemcpyHostToDevice, stream);
-        if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaMemcpyAsync(grad H2D)");
-    }
-    s = launch_step(ctx, hp, stream);
-    if (s != CAME_OK) return s;
-    if (host_params_out) {
-        for (int i = 0; i < ctx->n; ++i) {
-            if (!host_params_out[i]) continue;
+    const StepConsts hc = make_consts(*hp);
+    cudaError_t e;
+#define CAME_CK(call, what) do { e = (call); if (e != cudaSuccess) return cuda_fail(ctx, e, what); } while (0)
+    // Three-stage pipeline over groups of consecutive tensors (tensors are independent):
+    // upload gradients of group k+1 | step group k | download parameters of group k-1.
+    // The copy streams start after everything already queued on the caller's stream, and the
+    // caller's stream ends up waiting for the last download.
+    CAME_CK(cudaEventRecord(ctx->ev_start, stream), "cudaEventRecord");
+    CAME_CK(cudaStreamWaitEvent(ctx->s_up, ctx->ev_start, 0), "cudaStreamWaitEvent");
+    CAME_CK(cudaStreamWaitEvent(ctx->s_down, ctx->ev_start, 0), "cudaStreamWaitEvent");
+    const size_t ng = ctx->host_groups.size();
+    for (size_t k = 0; k < ng; ++k) {
+        const Group& g = ctx->host_groups[k];
+        for (int i = g.t0; i < g.t1; ++i) {
             const came_tensor& x = ctx->tensors[i];
-            const size_t bytes = static_cast<size_t>(x.rows) * x.cols * 4;
-            const cudaError_t e = cudaMemcpyAsync(host_params_out[i], x.param, bytes,
-                                                  cudaMemcpyDeviceToHost, stream);
-            if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaMemcpyAsync(param D2H)");
+            const size_t bytes = static_cast<size_t>(x.rows) * x.cols * (x.grad_dtype == CAME_BF16 ? 2 : 4);
+            CAME_CK(cudaMemcpyAsync(const_cast<void*>(x.grad), host_grads[i], bytes,
+                                    cudaMemcpyHostToDevice, ctx->s_up), "cudaMemcpyAsync(grad H2D)");
+        }
+        CAME_CK(cudaEventRecord(ctx->ev_up[k], ctx->s_up), "cudaEventRecord");
+    }
+    for (size_t k = 0; k < ng; ++k) {
+        const Group& g = ctx->host_groups[k];
+        CAME_CK(cudaStreamWaitEvent(stream, ctx->ev_up[k], 0), "cudaStreamWaitEvent");
+        launch_range(ctx, hc, stream, g, nullptr);
+        CAME_CK(cudaGetLastError(), "kernel launch");
+        if (host_params_out) {
+            CAME_CK(cudaEventRecord(ctx->ev_done[k], stream), "cudaEventRecord");
+            CAME_CK(cudaStreamWaitEvent(ctx->s_down, ctx->ev_done[k], 0), "cudaStreamWaitEvent");
+            for (int i = g.t0; i < g.t1; ++i) {
+                if (!host_params_out[i]) continue;
+                const came_tensor& x = ctx->tensors[i];
+                const size_t bytes = static_cast<size_t>(x.rows) * x.cols * 4;
+                CAME_CK(cudaMemcpyAsync(host_params_out[i], x.param, bytes, cudaMemcpyDeviceToHost,
+                                        ctx->s_down), "cudaMemcpyAsync(param D2H)");
+            }
         }
     }
+    CAME_CK(cudaEventRecord(ctx->ev_all_down, ctx->s_down), "cudaEventRecord");
+    CAME_CK(cudaStreamWaitEvent(stream, ctx->ev_all_down, 0), "cudaStreamWaitEvent");
+#undef CAME_CK
+    ctx->n_intervals = 0;
+    ctx->last_step = hp->step;
     return CAME_OK;
 }
 

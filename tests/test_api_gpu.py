@@ -259,3 +259,43 @@ def test_cuda_graph_replay_matches_eager_launches(env):
     torch.cuda.synchronize()
     binding.came_destroy(ctx)
     assert _same(a.snapshot(), b.snapshot())
+
+
+def test_grouped_schedule_and_pipelined_host_step_are_bit_identical(env):
+    """Scheduling knobs change launch order only: running group by group, or pipelining the
+    host-buffer step over several groups, must reproduce the one-grid-per-phase result exactly."""
+    torch, binding = env
+    ref = Buffers(torch, binding, W_ODD, 15)
+    ctx = binding.came_create(ref.descs)
+    _run_steps(torch, binding, ref, ctx, 15, 1, 3)
+    binding.came_destroy(ctx)
+    want = ref.snapshot()
+
+    binding.came_tune(binding.CAME_TUNE_SCHED_GROUP_BYTES, 100_000)     # ~ one or two tensors per group
+    try:
+        a = Buffers(torch, binding, W_ODD, 15)
+        ctx = binding.came_create(a.descs)
+        _run_steps(torch, binding, a, ctx, 15, 1, 3)
+        binding.came_destroy(ctx)
+    finally:
+        binding.came_tune(binding.CAME_TUNE_SCHED_GROUP_BYTES, 0)
+    assert _same(want, a.snapshot())
+
+    binding.came_tune(binding.CAME_TUNE_HOST_GROUP_BYTES, 50_000)
+    try:
+        b = Buffers(torch, binding, W_ODD, 15)
+        ctx = binding.came_create(b.descs)
+        stream = torch.cuda.current_stream().cuda_stream
+        outs = [torch.empty(t.numel, dtype=torch.float32).pin_memory() for t in W_ODD.tensors]
+        for step in (1, 2, 3):
+            hg = [to_torch_grad(torch, synth.make_grad(W_ODD, 15, i, step), "cpu").reshape(-1).pin_memory()
+                  for i in range(len(W_ODD.tensors))]
+            binding.came_step_host(ctx, binding.make_hparams(step, **HP), [g.data_ptr() for g in hg],
+                                   [o.data_ptr() for o in outs], stream)
+            torch.cuda.current_stream().synchronize()      # the caller's stream alone is enough
+        binding.came_destroy(ctx)
+    finally:
+        binding.came_tune(binding.CAME_TUNE_HOST_GROUP_BYTES, 0)
+    assert _same(want, b.snapshot())
+    for o, p in zip(outs, b.p):
+        assert bool((o == p.cpu()).all())
