@@ -139,7 +139,7 @@ enum {
     CAME_Q_STREAM_BYTES = 2,     /* algorithmic bytes per step when no tensor stays on chip      */
     CAME_Q_COMPULSORY_BYTES = 3, /* floor: g, m, theta read once; m, theta written once          */
     CAME_Q_WORKSPACE_BYTES = 4,  /* device bytes the context allocated                           */
-    CAME_Q_NUM_TILES = 5,        /* matrix tiles in the launch plan                              */
+    CAME_Q_NUM_TILES = 5,        /* tiles in the launch plan (matrix tiles + vector chunks)      */
     CAME_Q_LAUNCHES_PER_STEP = 6,/* kernels one came_step enqueues                               */
     CAME_Q_LAST_STEP = 7,        /* last step accepted (0 before the first)                      */
     CAME_Q_NUM_PHASES = 8,       /* entries came_get_phase_ms reports                            */

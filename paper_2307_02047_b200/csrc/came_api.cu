@@ -14,16 +14,14 @@
 
 using came::TensorDev;
 using came::Tile;
-using came::VChunk;
 using came::StepConsts;
 
 namespace {
 
-constexpr int kMaxPhases = 7;
+constexpr int kMaxPhases = 5;
 constexpr int kProfSlots = 128;        // profiled steps kept for averaging
 const char* const kPhaseNames[kMaxPhases] = {
-    "vec_second_moment", "p1_reduce_g2", "p2_sum_u2", "p3_momentum_instability", "p4_apply",
-    "p34_adafactor_apply", "vec_apply"};
+    "p1_reduce_g2", "p2_sum_u2", "p3_momentum_instability", "p4_apply", "p34_adafactor_apply"};
 
 thread_local std::string g_create_error;
 long long g_tile_elems_override = 0;   // came_tune(CAME_TUNE_TILE_ELEMS)
@@ -83,8 +81,8 @@ Plan plan_tensor(long long rows, long long cols, int ndim, int dtype, bool align
 
 }  // namespace
 
-// A run of consecutive tensors handled together: [t0, t1) with their tiles and vector chunks.
-struct Group { int t0, t1, tile0, tile1, chunk0, chunk1; };
+// A run of consecutive tensors handled together: [t0, t1) and their tiles.
+struct Group { int t0, t1, tile0, tile1; };
 
 struct came_ctx {
     int device = 0;
@@ -97,9 +95,8 @@ struct came_ctx {
     bool pinned_used[2] = {false, false};
     int pinned_next = 0;
     Tile* d_tiles = nullptr;
-    VChunk* d_chunks = nullptr;
-    int n_tiles = 0, n_chunks = 0;
-    std::vector<int> tile_begin, chunk_begin;   // [n+1] first tile / vector chunk of each tensor
+    int n_tiles = 0;                            // matrix tiles and vector chunks
+    std::vector<int> tile_begin;                // [n+1] first tile of each tensor
     std::vector<Group> sched_groups;            // device-resident step: launch order (empty = one grid)
     std::vector<Group> host_groups;             // host-buffer step: pipeline stages
     cudaStream_t s_up = nullptr, s_down = nullptr;   // copy streams of the host-buffer step
@@ -212,7 +209,6 @@ void free_ctx(came_ctx* ctx)
     cudaSetDevice(ctx->device);
     cudaFree(ctx->d_table);
     cudaFree(ctx->d_tiles);
-    cudaFree(ctx->d_chunks);
     cudaFree(ctx->d_ws);
     for (int k = 0; k < 2; ++k) {
         if (ctx->pinned_table[k]) cudaFreeHost(ctx->pinned_table[k]);
@@ -256,14 +252,9 @@ int launch_range(const came_ctx* ctx, const StepConsts& hc, cudaStream_t stream,
 {
     int iv = 0;
     auto mark = [&](int slot) { if (ev) cudaEventRecord(ev[slot], stream); };
-    const int nt = g.tile1 - g.tile0, nc = g.chunk1 - g.chunk0;
+    const int nt = g.tile1 - g.tile0;
     const Tile* tiles = ctx->d_tiles + g.tile0;
-    const VChunk* chunks = ctx->d_chunks + g.chunk0;
     mark(0);
-    if (nc > 0) {
-        came::k_vec_second_moment<<<nc, came::kThreads, 0, stream>>>(ctx->d_table, chunks, hc);
-        mark(++iv);
-    }
     if (nt > 0) {
         came::k_p1_reduce_g2<<<nt, came::kThreads, 0, stream>>>(ctx->d_table, tiles, nt, 0, hc);
         mark(++iv);
@@ -279,10 +270,6 @@ int launch_range(const came_ctx* ctx, const StepConsts& hc, cudaStream_t stream,
             mark(++iv);
         }
     }
-    if (nc > 0) {
-        came::k_vec_apply<<<nc, came::kThreads, 0, stream>>>(ctx->d_table, chunks, hc);
-        mark(++iv);
-    }
     return iv;
 }
 
@@ -292,7 +279,7 @@ came_status launch_step(came_ctx* ctx, const came_hparams* hp, cudaStream_t stre
     if (ctx->sched_groups.empty()) {
         const bool prof = ctx->profiling && !ctx->prof_ev.empty();
         cudaEvent_t* ev = prof ? &ctx->prof_ev[(ctx->prof_count % kProfSlots) * (kMaxPhases + 1)] : nullptr;
-        const Group all{0, ctx->n, 0, ctx->n_tiles, 0, ctx->n_chunks};
+        const Group all{0, ctx->n, 0, ctx->n_tiles};
         ctx->n_intervals = launch_range(ctx, hc, stream, all, ev);
         if (prof) ++ctx->prof_count;
     } else {
@@ -317,8 +304,7 @@ std::vector<Group> make_groups(const came_ctx* ctx, long long limit, F bytes_of)
     for (int i = 0; i < ctx->n; ++i) {
         acc += bytes_of(ctx->tensors[i]);
         if (acc >= limit || i == ctx->n - 1) {
-            out.push_back(Group{t0, i + 1, ctx->tile_begin[t0], ctx->tile_begin[i + 1],
-                                ctx->chunk_begin[t0], ctx->chunk_begin[i + 1]});
+            out.push_back(Group{t0, i + 1, ctx->tile_begin[t0], ctx->tile_begin[i + 1]});
             t0 = i + 1;
             acc = 0;
         }
@@ -423,9 +409,7 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
     }
     std::vector<Plan> plans(n);
     ctx->tile_begin.assign(n + 1, 0);
-    ctx->chunk_begin.assign(n + 1, 0);
     std::vector<Tile> tiles;
-    std::vector<VChunk> chunks;
     size_t ws = 0;
     auto take = [&](size_t bytes) { const size_t off = ws; ws += (bytes + 255) / 256 * 256; return off; };
     struct Off { size_t colpart, colpart2, rowpart, blocksum, usq, cnt, scal, rowscale, colscale; };
@@ -463,7 +447,7 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
             ctx->state_bytes += 4 * (conf ? 3 : 2) * numel;
             ctx->stream_bytes += numel * (sg + (conf ? 32 : 24));
             ctx->comp_bytes += numel * (sg + (conf ? 32 : 24));
-            for (int c = 0; c < p.n_parts; ++c) chunks.push_back(VChunk{i, c});
+            for (int c = 0; c < p.n_parts; ++c) tiles.push_back(Tile{i, c, 0});
             offs[i].colpart = offs[i].colpart2 = offs[i].rowpart = offs[i].blocksum = 0;
             offs[i].rowscale = offs[i].colscale = 0;
         }
@@ -471,14 +455,12 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
         offs[i].cnt = take(sizeof(unsigned) * p.counters());
         offs[i].scal = take(sizeof(float) * 4);
         ctx->tile_begin[i + 1] = static_cast<int>(tiles.size());
-        ctx->chunk_begin[i + 1] = static_cast<int>(chunks.size());
-        if (tiles.size() > (1u << 30) || chunks.size() > (1u << 30)) {
+        if (tiles.size() > (1u << 30)) {
             delete ctx;
             return fail(nullptr, CAME_ERR_SHAPE, "too many tiles");
         }
     }
     ctx->n_tiles = static_cast<int>(tiles.size());
-    ctx->n_chunks = static_cast<int>(chunks.size());
     ctx->ws_bytes = ws;
     ctx->table_bytes = sizeof(TensorDev) * n;
 
@@ -493,11 +475,6 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
         CAME_TRY(cudaMalloc(&ctx->d_tiles, sizeof(Tile) * tiles.size()), "cudaMalloc(tiles)");
         CAME_TRY(cudaMemcpy(ctx->d_tiles, tiles.data(), sizeof(Tile) * tiles.size(),
                             cudaMemcpyHostToDevice), "cudaMemcpy(tiles)");
-    }
-    if (ctx->n_chunks) {
-        CAME_TRY(cudaMalloc(&ctx->d_chunks, sizeof(VChunk) * chunks.size()), "cudaMalloc(chunks)");
-        CAME_TRY(cudaMemcpy(ctx->d_chunks, chunks.data(), sizeof(VChunk) * chunks.size(),
-                            cudaMemcpyHostToDevice), "cudaMemcpy(chunks)");
     }
     for (int k = 0; k < 2; ++k) {
         CAME_TRY(cudaMallocHost(&ctx->pinned_table[k], ctx->table_bytes), "cudaMallocHost(table)");
@@ -662,15 +639,14 @@ came_status came_query(const came_ctx* ctx, int32_t what, int64_t* out)
         case CAME_Q_STREAM_BYTES: *out = ctx->stream_bytes; break;
         case CAME_Q_COMPULSORY_BYTES: *out = ctx->comp_bytes; break;
         case CAME_Q_WORKSPACE_BYTES:
-            *out = static_cast<int64_t>(ctx->ws_bytes + ctx->table_bytes + sizeof(Tile) * ctx->n_tiles +
-                                        sizeof(VChunk) * ctx->n_chunks);
+            *out = static_cast<int64_t>(ctx->ws_bytes + ctx->table_bytes + sizeof(Tile) * ctx->n_tiles);
             break;
         case CAME_Q_NUM_TILES: *out = ctx->n_tiles; break;
         case CAME_Q_LAUNCHES_PER_STEP:
-            *out = (ctx->n_tiles ? (ctx->adafactor ? 3 : 4) : 0) + (ctx->n_chunks ? 2 : 0); break;
+            *out = ctx->adafactor ? 3 : 4; break;
         case CAME_Q_LAST_STEP: *out = ctx->last_step; break;
         case CAME_Q_NUM_PHASES:
-            *out = (ctx->n_tiles ? (ctx->adafactor ? 3 : 4) : 0) + (ctx->n_chunks ? 2 : 0); break;
+            *out = ctx->adafactor ? 3 : 4; break;
         case CAME_Q_MATRIX_NUMEL: *out = ctx->matrix_numel; break;
         default: return CAME_ERR_UNSUPPORTED;
     }
@@ -721,11 +697,10 @@ came_status came_get_phase_ms(came_ctx* ctx, float* out_ms, int32_t cap, int32_t
 const char* came_phase_name(const came_ctx* ctx, int32_t phase)
 {
     if (!ctx || phase < 0) return "";
-    // phases are reported in launch order; vectors-only or matrices-only contexts skip some
+    // phases are reported in launch order
+    const bool ada = ctx->adafactor;
+    const bool has[kMaxPhases] = {true, true, !ada, !ada, ada};
     int idx = 0;
-    const bool mat = ctx->n_tiles > 0, ada = ctx->adafactor;
-    const bool has[kMaxPhases] = {ctx->n_chunks > 0, mat, mat, mat && !ada, mat && !ada, mat && ada,
-                                  ctx->n_chunks > 0};
     for (int k = 0; k < kMaxPhases; ++k) {
         if (!has[k]) continue;
         if (idx == phase) return kPhaseNames[k];

@@ -3,7 +3,7 @@
 // One step of Algorithm 2 has three grid-wide data dependencies per tensor
 // (r,c need all of g; the clip factor needs all of u; S needs all of U), so a
 // matrix is streamed in four phases, each one kernel over a multi-tensor tile
-// list:
+// list (vectors ride along as extra tiles of P1 and P3):
 //   P1  g            -> row/column sums of g^2        -> r_t, c_t, sqrt(1^T r_t)
 //   P2  g, r, c      -> sum of u^2                    -> clip factor kappa (Eq. 1)
 //   P3  g, m, r, c   -> m_t, row/column sums of (uhat - m_{t-1})^2 -> R_t, C_t, sqrt(1^T R_t)
@@ -44,7 +44,8 @@ namespace came {
 #endif
 
 constexpr int kThreads = 256;
-constexpr int kVecChunk = 4096;       // vector elements per block in the vector kernels
+constexpr int kVecPerThread = 4;
+constexpr int kVecChunk = kThreads * kVecPerThread;   // vector elements per tile (one block)
 constexpr int kColGroup = 16;         // row blocks per group in the two-level column reduction
 
 enum Kind : int { kF32x4 = 0, kBF16x8 = 1, kF32x1 = 2, kBF16x1 = 3 };
@@ -80,8 +81,7 @@ struct TensorDev {
     unsigned     flags;
 };
 
-struct Tile { int tensor, rb, cb; };
-struct VChunk { int tensor, chunk; };
+struct Tile { int tensor, rb, cb; };   // vectors: rb = chunk of kVecChunk elements, cb = 0
 
 struct StepConsts {
     float beta1, omb1, b1sq;
@@ -852,6 +852,87 @@ __device__ __forceinline__ void p34_adafactor_tile(const TensorDev& d, int rb, i
 }
 
 // ---------------------------------------------------------------------------
+// vectors: the unfactored path.  A vector is cut into chunks of kVecChunk elements that ride
+// in the tile list: the first half runs in P1's grid, the second (after kappa) in P3's.
+// Each thread owns kVecPerThread elements and issues all their loads before using any.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ float load_grad_scalar(const TensorDev& d, long long i)
+{
+    if (d.kind == kBF16x1 || d.kind == kBF16x8)
+        return __uint_as_float(static_cast<uint32_t>(__ldg(static_cast<const uint16_t*>(d.g) + i)) << 16);
+    return __ldg(static_cast<const float*>(d.g) + i);
+}
+
+// v_t = beta2 v + (1-beta2)(g^2 + eps1);  partial sum of u^2 = g^2 / v_t;  kappa when complete
+__device__ __forceinline__ void vec_second_moment_chunk(const TensorDev& d, int chunk,
+                                                        const StepConsts& hc, Shared& sm)
+{
+    const long long i0 = static_cast<long long>(chunk) * kVecChunk + threadIdx.x;
+    float g[kVecPerThread], v[kVecPerThread];
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+        const long long i = i0 + k * kThreads;
+        const bool ok = i < d.rows;
+        g[k] = ok ? load_grad_scalar(d, i) * hc.gscale : 0.f;
+        v[k] = ok ? d.r[i] : 1.f;
+    }
+    float acc = 0.f;
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+        const long long i = i0 + k * kThreads;
+        if (i < d.rows) {
+            const float vn = fmaf(hc.beta2, v[k], hc.omb2 * fmaf(g[k], g[k], hc.eps1));
+            d.r[i] = vn;
+            const float u = g[k] * __frsqrt_rn(vn);
+            acc = fmaf(u, u, acc);
+        }
+    }
+    acc = block_sum(acc, sm);
+    finalize_kappa(d, chunk, acc, hc.clip_d, sm);
+}
+
+// uhat, m_t, S_t, theta_t (S and the confidence term skipped for kFlagVecNoConf)
+__device__ __forceinline__ void vec_apply_chunk(const TensorDev& d, int chunk, const StepConsts& hc)
+{
+    const long long i0 = static_cast<long long>(chunk) * kVecChunk + threadIdx.x;
+    const float kappa = d.scal[1];
+    const float wd = (d.flags & kFlagNoWd) ? 0.f : hc.wd;
+    const bool noconf = (d.flags & kFlagVecNoConf) != 0;
+    float g[kVecPerThread], v[kVecPerThread], mo[kVecPerThread], th[kVecPerThread], S[kVecPerThread];
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+        const long long i = i0 + k * kThreads;
+        const bool ok = i < d.rows;
+        g[k] = ok ? load_grad_scalar(d, i) * hc.gscale : 0.f;
+        v[k] = ok ? d.r[i] : 1.f;
+        mo[k] = ok ? d.m[i] : 0.f;
+        th[k] = ok ? d.p[i] : 0.f;
+        S[k] = (ok && !noconf) ? d.R[i] : 1.f;
+    }
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+        const long long i = i0 + k * kThreads;
+        if (i < d.rows) {
+            const float uh = (g[k] * __frsqrt_rn(v[k])) * kappa;
+            const float e = uh - mo[k];
+            const float mn = fmaf(hc.omb1, e, mo[k]);
+            d.m[i] = mn;
+            float dir;
+            if (noconf) {
+                dir = mn;
+            } else {
+                const float Sn = fmaf(hc.beta3, S[k], hc.omb3 * fmaf(hc.b1sq * e, e, hc.eps2));
+                d.R[i] = Sn;
+                dir = mn * __frsqrt_rn(Sn);
+            }
+            const float tn = fmaf(-hc.lr, fmaf(wd, th[k], dir), th[k]);
+            d.p[i] = tn;
+            if (d.p_bf16) d.p_bf16[i] = static_cast<uint16_t>(pack_bf16x2(tn, 0.f) & 0xffffu);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
 // kernels: one block per tile, block-uniform dispatch on the tensor's kind
 // ---------------------------------------------------------------------------
 #define CAME_DISPATCH(FN, ...)                                         \
@@ -875,6 +956,7 @@ k_p1_reduce_g2(const TensorDev* __restrict__ T, const Tile* __restrict__ tiles, 
     __shared__ Shared sm;
     const Tile t = fetch_tile(tiles, ntiles, reverse);
     const TensorDev d = T[t.tensor];       // by value: descriptor fields live in registers
+    if (d.ndim == 1) { vec_second_moment_chunk(d, t.rb, hc, sm); return; }
     CAME_DISPATCH(p1_tile, d, t.rb, t.cb, hc, sm)
 }
 
@@ -885,6 +967,7 @@ k_p2_sum_u2(const TensorDev* __restrict__ T, const Tile* __restrict__ tiles, int
     __shared__ Shared sm;
     const Tile t = fetch_tile(tiles, ntiles, reverse);
     const TensorDev d = T[t.tensor];
+    if (d.ndim == 1) return;               // vectors have no second reduction pass
     CAME_DISPATCH(p2_tile, d, t.rb, t.cb, hc, sm)
 }
 
@@ -895,6 +978,7 @@ k_p3_momentum_instability(const TensorDev* __restrict__ T, const Tile* __restric
     __shared__ Shared sm;
     const Tile t = fetch_tile(tiles, ntiles, reverse);
     const TensorDev d = T[t.tensor];
+    if (d.ndim == 1) { vec_apply_chunk(d, t.rb, hc); return; }
     CAME_DISPATCH(p3_tile, d, t.rb, t.cb, hc, sm)
 }
 
@@ -904,6 +988,7 @@ k_p4_apply(const TensorDev* __restrict__ T, const Tile* __restrict__ tiles, int 
 {
     const Tile t = fetch_tile(tiles, ntiles, reverse);
     const TensorDev d = T[t.tensor];
+    if (d.ndim == 1) return;               // vectors finished in P3's grid
     CAME_DISPATCH(p4_tile, d, t.rb, t.cb, hc)
 }
 
@@ -913,72 +998,8 @@ k_p34_adafactor_apply(const TensorDev* __restrict__ T, const Tile* __restrict__ 
 {
     const Tile t = fetch_tile(tiles, ntiles, reverse);
     const TensorDev d = T[t.tensor];
+    if (d.ndim == 1) { vec_apply_chunk(d, t.rb, hc); return; }
     CAME_DISPATCH(p34_adafactor_tile, d, t.rb, t.cb, hc)
-}
-
-// ---------------------------------------------------------------------------
-// vectors: the unfactored path, two kernels around the clip barrier
-// ---------------------------------------------------------------------------
-__device__ __forceinline__ float load_grad_scalar(const TensorDev& d, long long i)
-{
-    if (d.kind == kBF16x1 || d.kind == kBF16x8)
-        return __uint_as_float(static_cast<uint32_t>(__ldg(static_cast<const uint16_t*>(d.g) + i)) << 16);
-    return __ldg(static_cast<const float*>(d.g) + i);
-}
-
-// VA: v_t = beta2 v + (1-beta2)(g^2 + eps1);  partial sums of u^2 = g^2 / v_t;  kappa
-__global__ void __launch_bounds__(kThreads)
-k_vec_second_moment(const TensorDev* __restrict__ T, const VChunk* __restrict__ chunks,
-                    StepConsts hc)
-{
-    __shared__ Shared sm;
-    const VChunk ck = chunks[blockIdx.x];
-    const TensorDev& d = T[ck.tensor];
-    const long long i0 = static_cast<long long>(ck.chunk) * kVecChunk;
-    const long long i1 = min(d.rows, i0 + kVecChunk);
-    float acc = 0.f;
-    for (long long i = i0 + threadIdx.x; i < i1; i += kThreads) {
-        const float g = load_grad_scalar(d, i) * hc.gscale;
-        const float vn = fmaf(hc.beta2, d.r[i], hc.omb2 * fmaf(g, g, hc.eps1));
-        d.r[i] = vn;
-        const float u = g * __frsqrt_rn(vn);
-        acc = fmaf(u, u, acc);
-    }
-    acc = block_sum(acc, sm);
-    finalize_kappa(d, ck.chunk, acc, hc.clip_d, sm);
-}
-
-// VB: uhat, m_t, S_t, theta_t
-__global__ void __launch_bounds__(kThreads)
-k_vec_apply(const TensorDev* __restrict__ T, const VChunk* __restrict__ chunks, StepConsts hc)
-{
-    const VChunk ck = chunks[blockIdx.x];
-    const TensorDev& d = T[ck.tensor];
-    const long long i0 = static_cast<long long>(ck.chunk) * kVecChunk;
-    const long long i1 = min(d.rows, i0 + kVecChunk);
-    const float kappa = d.scal[1];
-    const float wd = (d.flags & kFlagNoWd) ? 0.f : hc.wd;
-    const bool noconf = (d.flags & kFlagVecNoConf) != 0;
-    for (long long i = i0 + threadIdx.x; i < i1; i += kThreads) {
-        const float g = load_grad_scalar(d, i) * hc.gscale;
-        const float uh = (g * __frsqrt_rn(d.r[i])) * kappa;
-        const float mo = d.m[i];
-        const float e = uh - mo;
-        const float mn = fmaf(hc.omb1, e, mo);
-        d.m[i] = mn;
-        const float th = d.p[i];
-        float dir;
-        if (noconf) {
-            dir = mn;
-        } else {
-            const float Sn = fmaf(hc.beta3, d.R[i], hc.omb3 * fmaf(hc.b1sq * e, e, hc.eps2));
-            d.R[i] = Sn;
-            dir = mn * __frsqrt_rn(Sn);
-        }
-        const float tn = fmaf(-hc.lr, fmaf(wd, th, dir), th);
-        d.p[i] = tn;
-        if (d.p_bf16) d.p_bf16[i] = static_cast<uint16_t>(pack_bf16x2(tn, 0.f) & 0xffffu);
-    }
 }
 
 }  // namespace came

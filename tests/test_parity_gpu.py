@@ -121,7 +121,7 @@ def test_adafactor_mode_needs_no_instability_state(env):
         binding.came_create(descs)                      # Algorithm 2 needs R and C
     assert e.value.status == 1
     ctx = binding.came_create(descs, flags=binding.CAME_CREATE_ADAFACTOR)
-    assert binding.came_query(ctx, binding.CAME_Q_LAUNCHES_PER_STEP) == 5
+    assert binding.came_query(ctx, binding.CAME_Q_LAUNCHES_PER_STEP) == 3
     binding.came_step(ctx, binding.make_hparams(1, **w.hparams), None,
                       torch.cuda.current_stream().cuda_stream)
     torch.cuda.synchronize()
