@@ -249,8 +249,12 @@ enum {
                                          tensors (about this many bytes of g, m and theta) before
                                          the next group, instead of one grid per phase over all
                                          tensors; per-phase timing is then not reported.  0 = off. */
-    CAME_TUNE_HOST_GROUP_BYTES = 2    /* bytes of gradients + parameters per pipeline stage of
+    CAME_TUNE_HOST_GROUP_BYTES = 2,   /* bytes of gradients + parameters per pipeline stage of
                                          came_step_host (default 1 GiB) */
+    CAME_TUNE_PDL = 3                 /* 1 (default): phase kernels use programmatic dependent
+                                         launch, so a phase's blocks are scheduled during the
+                                         previous phase's tail; 0: plain stream order.  Read at
+                                         every step. */
 };
 came_status came_tune(int32_t key, int64_t value);
 

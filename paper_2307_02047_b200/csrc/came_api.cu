@@ -25,6 +25,7 @@ const char* const kPhaseNames[kMaxPhases] = {
 
 thread_local std::string g_create_error;
 long long g_tile_elems_override = 0;   // came_tune(CAME_TUNE_TILE_ELEMS)
+bool g_use_pdl = true;                 // came_tune(CAME_TUNE_PDL)
 long long g_sched_group_bytes = 0;     // came_tune(CAME_TUNE_SCHED_GROUP_BYTES); 0 = one group
 long long g_host_group_bytes = 1ll << 30;   // came_tune(CAME_TUNE_HOST_GROUP_BYTES)
 
@@ -245,6 +246,24 @@ came_status upload_table(came_ctx* ctx, cudaStream_t stream)
     return CAME_OK;
 }
 
+// Launch one phase kernel with programmatic stream serialisation (see pdl_* in the kernels).
+template <typename K>
+void launch_phase(K kernel, int grid, cudaStream_t stream, const TensorDev* table, const Tile* tiles,
+                  int ntiles, int reverse, const StepConsts& hc)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid));
+    cfg.blockDim = dim3(came::kThreads);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = g_use_pdl ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kernel, table, tiles, ntiles, reverse, hc);
+}
+
 // Enqueue the kernels of one step for the tensors of `g` (all phases, in dependency order).
 // `ev` (may be NULL) receives one event before the first kernel and one after each kernel.
 int launch_range(const came_ctx* ctx, const StepConsts& hc, cudaStream_t stream, const Group& g,
@@ -256,17 +275,17 @@ int launch_range(const came_ctx* ctx, const StepConsts& hc, cudaStream_t stream,
     const Tile* tiles = ctx->d_tiles + g.tile0;
     mark(0);
     if (nt > 0) {
-        came::k_p1_reduce_g2<<<nt, came::kThreads, 0, stream>>>(ctx->d_table, tiles, nt, 0, hc);
+        launch_phase(came::k_p1_reduce_g2, nt, stream, ctx->d_table, tiles, nt, 0, hc);
         mark(++iv);
-        came::k_p2_sum_u2<<<nt, came::kThreads, 0, stream>>>(ctx->d_table, tiles, nt, 1, hc);
+        launch_phase(came::k_p2_sum_u2, nt, stream, ctx->d_table, tiles, nt, 1, hc);
         mark(++iv);
         if (ctx->adafactor) {
-            came::k_p34_adafactor_apply<<<nt, came::kThreads, 0, stream>>>(ctx->d_table, tiles, nt, 0, hc);
+            launch_phase(came::k_p34_adafactor_apply, nt, stream, ctx->d_table, tiles, nt, 0, hc);
             mark(++iv);
         } else {
-            came::k_p3_momentum_instability<<<nt, came::kThreads, 0, stream>>>(ctx->d_table, tiles, nt, 0, hc);
+            launch_phase(came::k_p3_momentum_instability, nt, stream, ctx->d_table, tiles, nt, 0, hc);
             mark(++iv);
-            came::k_p4_apply<<<nt, came::kThreads, 0, stream>>>(ctx->d_table, tiles, nt, 1, hc);
+            launch_phase(came::k_p4_apply, nt, stream, ctx->d_table, tiles, nt, 1, hc);
             mark(++iv);
         }
     }
@@ -346,6 +365,7 @@ came_status came_tune(int32_t key, int64_t value)
     switch (key) {
         case CAME_TUNE_TILE_ELEMS: g_tile_elems_override = value; break;
         case CAME_TUNE_SCHED_GROUP_BYTES: g_sched_group_bytes = value; break;
+        case CAME_TUNE_PDL: g_use_pdl = value != 0; break;
         case CAME_TUNE_HOST_GROUP_BYTES: g_host_group_bytes = value > 0 ? value : (1ll << 30); break;
         default: return CAME_ERR_UNSUPPORTED;
     }

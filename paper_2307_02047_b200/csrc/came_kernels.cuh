@@ -949,13 +949,24 @@ __device__ __forceinline__ Tile fetch_tile(const Tile* tiles, int ntiles, int re
     return tiles[reverse ? (ntiles - 1 - b) : b];
 }
 
+// Programmatic dependent launch: the phase kernels are launched with stream serialisation
+// relaxed, so the next phase's blocks may be scheduled while this phase's last blocks are still
+// running.  A block lets its dependents go at once (they hold no resources this grid still
+// needs: every block of this grid has started by then) and, after reading only the tile list
+// and the tensor table (written by copies, never by a kernel), waits for the whole previous
+// grid, memory included, before it touches anything a kernel produced.
+__device__ __forceinline__ void pdl_release_dependents() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void pdl_wait_for_previous_grid() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __global__ void __launch_bounds__(kThreads, CAME_P1_MINB)
 k_p1_reduce_g2(const TensorDev* __restrict__ T, const Tile* __restrict__ tiles, int ntiles,
                int reverse, StepConsts hc)
 {
     __shared__ Shared sm;
+    pdl_release_dependents();
     const Tile t = fetch_tile(tiles, ntiles, reverse);
     const TensorDev d = T[t.tensor];       // by value: descriptor fields live in registers
+    pdl_wait_for_previous_grid();
     if (d.ndim == 1) { vec_second_moment_chunk(d, t.rb, hc, sm); return; }
     CAME_DISPATCH(p1_tile, d, t.rb, t.cb, hc, sm)
 }
@@ -965,8 +976,10 @@ k_p2_sum_u2(const TensorDev* __restrict__ T, const Tile* __restrict__ tiles, int
             int reverse, StepConsts hc)
 {
     __shared__ Shared sm;
+    pdl_release_dependents();
     const Tile t = fetch_tile(tiles, ntiles, reverse);
     const TensorDev d = T[t.tensor];
+    pdl_wait_for_previous_grid();
     if (d.ndim == 1) return;               // vectors have no second reduction pass
     CAME_DISPATCH(p2_tile, d, t.rb, t.cb, hc, sm)
 }
@@ -976,8 +989,10 @@ k_p3_momentum_instability(const TensorDev* __restrict__ T, const Tile* __restric
                           int ntiles, int reverse, StepConsts hc)
 {
     __shared__ Shared sm;
+    pdl_release_dependents();
     const Tile t = fetch_tile(tiles, ntiles, reverse);
     const TensorDev d = T[t.tensor];
+    pdl_wait_for_previous_grid();
     if (d.ndim == 1) { vec_apply_chunk(d, t.rb, hc); return; }
     CAME_DISPATCH(p3_tile, d, t.rb, t.cb, hc, sm)
 }
@@ -986,8 +1001,10 @@ __global__ void __launch_bounds__(kThreads, CAME_P4_MINB)
 k_p4_apply(const TensorDev* __restrict__ T, const Tile* __restrict__ tiles, int ntiles,
            int reverse, StepConsts hc)
 {
+    pdl_release_dependents();
     const Tile t = fetch_tile(tiles, ntiles, reverse);
     const TensorDev d = T[t.tensor];
+    pdl_wait_for_previous_grid();
     if (d.ndim == 1) return;               // vectors finished in P3's grid
     CAME_DISPATCH(p4_tile, d, t.rb, t.cb, hc)
 }
@@ -996,8 +1013,10 @@ __global__ void __launch_bounds__(kThreads, 2)
 k_p34_adafactor_apply(const TensorDev* __restrict__ T, const Tile* __restrict__ tiles, int ntiles,
                       int reverse, StepConsts hc)
 {
+    pdl_release_dependents();
     const Tile t = fetch_tile(tiles, ntiles, reverse);
     const TensorDev d = T[t.tensor];
+    pdl_wait_for_previous_grid();
     if (d.ndim == 1) { vec_apply_chunk(d, t.rb, hc); return; }
     CAME_DISPATCH(p34_adafactor_tile, d, t.rb, t.cb, hc)
 }
