@@ -608,10 +608,10 @@ __device__ __forceinline__ void p2_tile(const TensorDev& d, int rb, int cb, cons
     const char* gp = static_cast<const char*>(d.g) +
                      ((q.row0 + q.ty) * d.cols + q.col) * grad_elem_bytes<KIND>();
     const float* ap = d.ws_rowscale + q.row0 + q.ty;
-    const float ssr = d.scal[0] * hc.gscale;          // sqrt(sum r) * gradient pre-scale
+    const float ssr = __ldcg(d.scal + 0) * hc.gscale;          // sqrt(sum r) * gradient pre-scale
     float b[VEC];
 #pragma unroll
-    for (int v = 0; v < VEC; ++v) b[v] = q.colok ? d.ws_colscale[q.col + v] : 0.f;
+    for (int v = 0; v < VEC; ++v) b[v] = q.colok ? __ldcg(d.ws_colscale + q.col + v) : 0.f;
     float acc = 0.f;
 
     for (long long rbase = q.row0 + q.ty; rbase < q.row1; rbase += static_cast<long long>(q.TY) * U) {
@@ -620,12 +620,12 @@ __device__ __forceinline__ void p2_tile(const TensorDev& d, int rb, int cb, cons
         const bool full = rbase + static_cast<long long>(U - 1) * q.TY < q.row1;
         if (full && q.colok) {
 #pragma unroll
-            for (int k = 0; k < U; ++k) { load_raw<KIND>(gp + k * stride, raw[k]); a[k] = ap[k * q.TY]; }
+            for (int k = 0; k < U; ++k) { load_raw<KIND>(gp + k * stride, raw[k]); a[k] = __ldcg(ap + k * q.TY); }
         } else {
 #pragma unroll
             for (int k = 0; k < U; ++k) {
                 if (q.colok && rbase + static_cast<long long>(k) * q.TY < q.row1) {
-                    load_raw<KIND>(gp + k * stride, raw[k]); a[k] = ap[k * q.TY];
+                    load_raw<KIND>(gp + k * stride, raw[k]); a[k] = __ldcg(ap + k * q.TY);
                 } else { zero_raw<KIND>(raw[k]); a[k] = 0.f; }
             }
         }
@@ -667,12 +667,12 @@ __device__ __forceinline__ void p3_tile(const TensorDev& d, int rb, int cb, cons
     float* mp = d.m + first;
     const float* ap = d.ws_rowscale + q.row0 + q.ty;
     float* const rowpart_seg = d.ws_rowpart + q.seg * d.rows;
-    const float ssr_k = d.scal[0] * d.scal[1] * hc.gscale;   // sqrt(sum r) * kappa * pre-scale
+    const float ssr_k = __ldcg(d.scal + 0) * __ldcg(d.scal + 1) * hc.gscale;   // sqrt(sum r) * kappa * pre-scale
     const float omb1 = hc.omb1;
     float b[VEC], cacc[VEC];
 #pragma unroll
     for (int v = 0; v < VEC; ++v) {
-        b[v] = q.colok ? d.ws_colscale[q.col + v] : 0.f;
+        b[v] = q.colok ? __ldcg(d.ws_colscale + q.col + v) : 0.f;
         cacc[v] = 0.f;
     }
 
@@ -685,7 +685,7 @@ __device__ __forceinline__ void p3_tile(const TensorDev& d, int rb, int cb, cons
             for (int k = 0; k < U; ++k) {
                 load_raw<KIND>(gp + k * gstride, raw[k]);
                 load_f<VEC>(mp + k * mstride, mo[k]);
-                a[k] = ap[k * q.TY];
+                a[k] = __ldcg(ap + k * q.TY);
             }
         } else {
 #pragma unroll
@@ -693,7 +693,7 @@ __device__ __forceinline__ void p3_tile(const TensorDev& d, int rb, int cb, cons
                 if (q.colok && rbase + static_cast<long long>(k) * q.TY < q.row1) {
                     load_raw<KIND>(gp + k * gstride, raw[k]);
                     load_f<VEC>(mp + k * mstride, mo[k]);
-                    a[k] = ap[k * q.TY];
+                    a[k] = __ldcg(ap + k * q.TY);
                 } else {
                     zero_raw<KIND>(raw[k]);
                     a[k] = 0.f;
@@ -747,12 +747,12 @@ __device__ __forceinline__ void p4_tile(const TensorDev& d, int rb, int cb, cons
     float* pp = d.p + first;
     uint16_t* hp16 = d.p_bf16 ? d.p_bf16 + first : nullptr;
     const float* ap = d.ws_rowscale + q.row0 + q.ty;
-    const float ssR = d.scal[2];
+    const float ssR = __ldcg(d.scal + 2);
     const float wd = (d.flags & kFlagNoWd) ? 0.f : hc.wd;
     const float nlr = -hc.lr;
     float B[VEC];
 #pragma unroll
-    for (int v = 0; v < VEC; ++v) B[v] = d.ws_colscale[q.col + v];
+    for (int v = 0; v < VEC; ++v) B[v] = __ldcg(d.ws_colscale + q.col + v);
 
     for (long long rbase = q.row0 + q.ty; rbase < q.row1; rbase += static_cast<long long>(q.TY) * U) {
         float mo[U][VEC], th[U][VEC], a[U];
@@ -762,7 +762,7 @@ __device__ __forceinline__ void p4_tile(const TensorDev& d, int rb, int cb, cons
             if (full || rbase + static_cast<long long>(k) * q.TY < q.row1) {
                 load_f<VEC>(mp + k * stride, mo[k]);
                 load_f<VEC>(pp + k * stride, th[k]);
-                a[k] = ap[k * q.TY];
+                a[k] = __ldcg(ap + k * q.TY);
             }
         }
 #pragma unroll
@@ -806,12 +806,12 @@ __device__ __forceinline__ void p34_adafactor_tile(const TensorDev& d, int rb, i
     float* pp = d.p + first;
     uint16_t* hp16 = d.p_bf16 ? d.p_bf16 + first : nullptr;
     const float* ap = d.ws_rowscale + q.row0 + q.ty;
-    const float ssr_k = d.scal[0] * d.scal[1] * hc.gscale;
+    const float ssr_k = __ldcg(d.scal + 0) * __ldcg(d.scal + 1) * hc.gscale;
     const float wd = (d.flags & kFlagNoWd) ? 0.f : hc.wd;
     const float nlr = -hc.lr, omb1 = hc.omb1;
     float b[VEC];
 #pragma unroll
-    for (int v = 0; v < VEC; ++v) b[v] = d.ws_colscale[q.col + v];
+    for (int v = 0; v < VEC; ++v) b[v] = __ldcg(d.ws_colscale + q.col + v);
 
     for (long long rbase = q.row0 + q.ty; rbase < q.row1; rbase += static_cast<long long>(q.TY) * U) {
         Raw<KIND> raw[U];
@@ -823,7 +823,7 @@ __device__ __forceinline__ void p34_adafactor_tile(const TensorDev& d, int rb, i
                 load_raw<KIND>(gp + k * gstride, raw[k]);
                 load_f<VEC>(mp + k * stride, mo[k]);
                 load_f<VEC>(pp + k * stride, th[k]);
-                a[k] = ap[k * q.TY];
+                a[k] = __ldcg(ap + k * q.TY);
             }
         }
 #pragma unroll
@@ -874,7 +874,7 @@ __device__ __forceinline__ void vec_second_moment_chunk(const TensorDev& d, int 
         const long long i = i0 + k * kThreads;
         const bool ok = i < d.rows;
         g[k] = ok ? load_grad_scalar(d, i) * hc.gscale : 0.f;
-        v[k] = ok ? d.r[i] : 1.f;
+        v[k] = ok ? __ldcg(d.r + i) : 1.f;
     }
     float acc = 0.f;
 #pragma unroll
@@ -895,7 +895,7 @@ __device__ __forceinline__ void vec_second_moment_chunk(const TensorDev& d, int 
 __device__ __forceinline__ void vec_apply_chunk(const TensorDev& d, int chunk, const StepConsts& hc)
 {
     const long long i0 = static_cast<long long>(chunk) * kVecChunk + threadIdx.x;
-    const float kappa = d.scal[1];
+    const float kappa = __ldcg(d.scal + 1);
     const float wd = (d.flags & kFlagNoWd) ? 0.f : hc.wd;
     const bool noconf = (d.flags & kFlagVecNoConf) != 0;
     float g[kVecPerThread], v[kVecPerThread], mo[kVecPerThread], th[kVecPerThread], S[kVecPerThread];
@@ -904,10 +904,10 @@ __device__ __forceinline__ void vec_apply_chunk(const TensorDev& d, int chunk, c
         const long long i = i0 + k * kThreads;
         const bool ok = i < d.rows;
         g[k] = ok ? load_grad_scalar(d, i) * hc.gscale : 0.f;
-        v[k] = ok ? d.r[i] : 1.f;
-        mo[k] = ok ? d.m[i] : 0.f;
-        th[k] = ok ? d.p[i] : 0.f;
-        S[k] = (ok && !noconf) ? d.R[i] : 1.f;
+        v[k] = ok ? __ldcg(d.r + i) : 1.f;
+        mo[k] = ok ? __ldcg(d.m + i) : 0.f;
+        th[k] = ok ? __ldcg(d.p + i) : 0.f;
+        S[k] = (ok && !noconf) ? __ldcg(d.R + i) : 1.f;
     }
 #pragma unroll
     for (int k = 0; k < kVecPerThread; ++k) {
