@@ -77,3 +77,47 @@ def test_bert_base_adafactor_mode(env):
     w = synth.workload("bert_base")
     _gate(run_paired(torch, binding, oracle, w, seed=2, steps=10, check_at=(1, 10), workers=WORKERS,
                      algorithm="adafactor"), "bert_base/adafactor")
+
+
+def test_matrix_with_more_than_2_pow_31_elements(env):
+    """Index arithmetic beyond 32 bits.  A matrix that is a K x K tiling of a small base block B
+    has, by Algorithm 2's own algebra, r and R equal to K times the base's (tiled), c and C
+    likewise, and v, u, m, S, theta equal to the base's in every copy (the factor K*K cancels
+    in r c / sum r).  So the oracle steps the base block and every copy of the 2.2 G-element
+    result is checked against it."""
+    torch, binding, oracle = env
+    import numpy as np
+    from tests.parity_util import err_signed, err_positive
+    nb, mb, K = 1024, 2056, 32                      # 32768 x 65792 = 2,155,872,256 elements
+    w = synth.workload(f"mat:{nb}x{mb}:bf16")
+    hp = dict(w.hparams)
+    p0 = synth.make_params(w, 41)[0]
+    dev = "cuda:0"
+    p = torch.from_numpy(p0).to(dev).repeat(K, K).contiguous()
+    g = torch.empty((nb * K, mb * K), dtype=torch.bfloat16, device=dev)
+    assert p.numel() > 2 ** 31
+    opt = binding.CameOptimizer([p], [g])
+    orc = oracle.OracleOptimizer([p0])
+    for step in (1, 2):
+        gb = synth.make_grad(w, 41, 0, step)
+        g.copy_(torch.from_numpy(gb.view(np.int16)).view(torch.bfloat16).to(dev).repeat(K, K))
+        opt.step(**hp)
+        orc.step([synth.widen(gb)], **hp)
+    torch.cuda.synchronize()
+    tol = TOL_STEP10
+    ref_p = torch.from_numpy(orc.p[0]).to(dev)
+    ref_m = torch.from_numpy(orc.m[0]).to(dev)
+    rms_p, rms_m = float(ref_p.square().mean().sqrt()), float(ref_m.square().mean().sqrt())
+    worst_p = worst_m = 0.0
+    for bi in range(K):                              # one block row at a time keeps temporaries small
+        blk_p = p[bi * nb:(bi + 1) * nb].view(nb, K, mb).double()
+        blk_m = opt.m[0][bi * nb:(bi + 1) * nb].view(nb, K, mb).double()
+        ep = ((blk_p - ref_p[:, None, :]).abs() / (ref_p.abs()[:, None, :] + rms_p)).max()
+        em = ((blk_m - ref_m[:, None, :]).abs() / (ref_m.abs()[:, None, :] + rms_m)).max()
+        worst_p, worst_m = max(worst_p, float(ep)), max(worst_m, float(em))
+    assert worst_p <= tol and worst_m <= tol, (worst_p, worst_m)
+    for got, want in ((opt.r[0], np.tile(orc.r[0], K) * K), (opt.c[0], np.tile(orc.c[0], K) * K),
+                      (opt.R[0], np.tile(orc.R[0], K) * K), (opt.C[0], np.tile(orc.C[0], K) * K)):
+        assert err_positive(got.cpu().numpy(), want) <= tol
+    print("PARITY >2^31", dict(p=worst_p, m=worst_m))
+    opt.close()

@@ -158,3 +158,41 @@ def test_grad_scale_is_validated(env):
         opt.step(**dict(w.hparams, grad_scale=-2.0))
     assert e.value.status == 5
     opt.close()
+
+
+# ---------------------------------------------------------------------------
+# degenerate inputs
+# ---------------------------------------------------------------------------
+def test_all_zero_gradients_stay_finite_and_match(env):
+    torch, binding, oracle = env
+    ts = (synth.mat("a", 130, 264), synth.mat("b", 1, 40), synth.vec("v", 300))
+    hp = dict(synth.PAPER_HPARAMS, weight_decay=0.01)
+    w = synth.Workload("zeros", ts, synth.BF16, "normal_fixed", 0.0, 0.0, (), 3, hp)   # scale 0: g == 0
+    res = run_paired(torch, binding, oracle, w, seed=27, steps=3, check_at=(1, 3))
+    _gate(res)
+
+
+def test_nan_in_one_tensor_does_not_touch_the_others(env):
+    """Tensors are independent in Algorithm 2; a non-finite gradient propagates inside its own
+    tensor only (the paper has no skip logic, and none is added)."""
+    torch, binding, oracle = env
+    ts = (synth.mat("a", 64, 264), synth.mat("b", 130, 520), synth.vec("v", 300), synth.vec("u", 77))
+    w = synth.Workload("nan", ts, synth.F32, "normal_fixed", 1e-3, 0.0, (), 2, dict(synth.PAPER_HPARAMS))
+    outs = []
+    for poison in (False, True):
+        p = [torch.from_numpy(x).cuda() for x in synth.make_params(w, 29)]
+        g = [torch.from_numpy(x).cuda() for x in synth.make_grads(w, 29, 1)]
+        if poison:
+            g[0][3, 5] = float("nan")
+            g[2][10] = float("inf")
+        opt = binding.CameOptimizer(p, g)
+        opt.step(**w.hparams)
+        opt.step(**w.hparams)
+        torch.cuda.synchronize()
+        outs.append([x.clone() for x in p] + [x.clone() for x in opt.m] + [opt.r[1].clone(), opt.C[1].clone()])
+        if poison:
+            assert not bool(p[0].isfinite().all()) and not bool(p[2].isfinite().all())
+        opt.close()
+    clean, dirty = outs
+    for i in (1, 3, 5, 7, 8, 9):                      # everything belonging to tensors 1 and 3
+        assert bool((clean[i] == dirty[i]).all())
