@@ -255,6 +255,9 @@ enum {
                                          launch, so a phase's blocks are scheduled during the
                                          previous phase's tail; 0: plain stream order.  Read at
                                          every step. */
+    , CAME_TUNE_F32_VEC8 = 4          /* 1 (default): fp32 gradients are read 8 per thread with
+                                         256-bit loads when rows are 32-byte aligned; 0: 4 per
+                                         thread (128-bit) */
 };
 came_status came_tune(int32_t key, int64_t value);
 

@@ -28,6 +28,7 @@ CAME_TUNE_TILE_ELEMS = 0
 CAME_TUNE_SCHED_GROUP_BYTES = 1
 CAME_TUNE_HOST_GROUP_BYTES = 2
 CAME_TUNE_PDL = 3
+CAME_TUNE_F32_VEC8 = 4
 
 EXPORTED = ["came_create", "came_step", "came_step_host", "came_destroy", "came_last_error",
             "came_status_string", "came_query", "came_set_profiling", "came_get_phase_ms",

@@ -29,6 +29,9 @@ bool g_use_pdl = true;                 // came_tune(CAME_TUNE_PDL)
 long long g_sched_group_bytes = 0;     // came_tune(CAME_TUNE_SCHED_GROUP_BYTES); 0 = one group
 long long g_host_group_bytes = 1ll << 30;   // came_tune(CAME_TUNE_HOST_GROUP_BYTES)
 
+bool g_f32_vec8 = true;                // came_tune(CAME_TUNE_F32_VEC8)
+inline bool g_f32_vec8_ok(bool bf) { return bf || g_f32_vec8; }
+
 struct Plan {
     int vec = 1, tx = 256, tr = 0, n_rb = 0, n_cb = 0, n_seg = 0, n_parts = 0, kind = 0;
     int n_grp = 0;
@@ -50,9 +53,18 @@ Plan plan_tensor(long long rows, long long cols, int ndim, int dtype, bool align
         p.n_parts = static_cast<int>(ceil_div(rows, came::kVecChunk));
         return p;
     }
-    const int vmax = bf ? 8 : 4;
-    p.vec = (cols % vmax == 0 && (!bf || aligned32)) ? vmax : 1;
-    p.kind = p.vec == 1 ? (bf ? came::kBF16x1 : came::kF32x1) : (bf ? came::kBF16x8 : came::kF32x4);
+    // 8 elements per thread (256-bit fp32 accesses) when rows start 32-byte aligned, else 4 for
+    // fp32 gradients (128-bit), else one element at a time
+    if (cols % 8 == 0 && aligned32 && g_f32_vec8_ok(bf)) {
+        p.vec = 8;
+        p.kind = bf ? came::kBF16x8 : came::kF32x8;
+    } else if (!bf && cols % 4 == 0) {
+        p.vec = 4;
+        p.kind = came::kF32x4;
+    } else {
+        p.vec = 1;
+        p.kind = bf ? came::kBF16x1 : came::kF32x1;
+    }
     const long long lanes = ceil_div(cols, p.vec);
     // widest block row whose padding wastes at most 1/8 of the lanes; else the least padding
     int best = 32;
@@ -366,6 +378,7 @@ came_status came_tune(int32_t key, int64_t value)
         case CAME_TUNE_TILE_ELEMS: g_tile_elems_override = value; break;
         case CAME_TUNE_SCHED_GROUP_BYTES: g_sched_group_bytes = value; break;
         case CAME_TUNE_PDL: g_use_pdl = value != 0; break;
+        case CAME_TUNE_F32_VEC8: g_f32_vec8 = value != 0; break;
         case CAME_TUNE_HOST_GROUP_BYTES: g_host_group_bytes = value > 0 ? value : (1ll << 30); break;
         default: return CAME_ERR_UNSUPPORTED;
     }
@@ -436,7 +449,8 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
     std::vector<Off> offs(n);
     for (int i = 0; i < n; ++i) {
         const came_tensor& x = t[i];
-        const bool a32 = aligned(x.param, 32) && aligned(x.m, 32);
+        const bool a32 = aligned(x.param, 32) && aligned(x.m, 32) &&
+                         (x.grad_dtype == CAME_BF16 || aligned(x.grad, 32));
         Plan p = plan_tensor(x.rows, x.cols, x.ndim, x.grad_dtype, a32, target);
         plans[i] = p;
         const long long numel = x.rows * x.cols;

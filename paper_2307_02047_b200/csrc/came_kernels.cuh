@@ -48,7 +48,7 @@ constexpr int kVecPerThread = 4;
 constexpr int kVecChunk = kThreads * kVecPerThread;   // vector elements per tile (one block)
 constexpr int kColGroup = 16;         // row blocks per group in the two-level column reduction
 
-enum Kind : int { kF32x4 = 0, kBF16x8 = 1, kF32x1 = 2, kBF16x1 = 3 };
+enum Kind : int { kF32x4 = 0, kBF16x8 = 1, kF32x1 = 2, kBF16x1 = 3, kF32x8 = 4 };
 
 struct TensorDev {
     float*       p;
@@ -103,6 +103,7 @@ constexpr unsigned kFlagVecNoConf = 1u << 1;
 template <int KIND> struct Traits;
 template <> struct Traits<kF32x4>  { static constexpr int VEC = 4; };
 template <> struct Traits<kBF16x8> { static constexpr int VEC = 8; };
+template <> struct Traits<kF32x8>  { static constexpr int VEC = 8; };   // 256-bit gradient loads
 template <> struct Traits<kF32x1>  { static constexpr int VEC = 1; };
 template <> struct Traits<kBF16x1> { static constexpr int VEC = 1; };
 
@@ -465,6 +466,7 @@ __device__ __forceinline__ Geo make_geo(const TensorDev& d, int rb, int cb)
 template <int KIND> struct Raw;
 template <> struct Raw<kF32x4>  { float4 v; };
 template <> struct Raw<kBF16x8> { uint4 v; };
+template <> struct Raw<kF32x8>  { float v[8]; };
 template <> struct Raw<kF32x1>  { float v; };
 template <> struct Raw<kBF16x1> { uint16_t v; };
 
@@ -473,6 +475,11 @@ __device__ __forceinline__ void load_raw(const char* p, Raw<KIND>& r)
 {
     if constexpr (KIND == kF32x4) r.v = __ldg(reinterpret_cast<const float4*>(p));
     else if constexpr (KIND == kBF16x8) r.v = __ldg(reinterpret_cast<const uint4*>(p));
+    else if constexpr (KIND == kF32x8) {
+        asm volatile("ld.global.nc.L1::no_allocate.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                     : "=f"(r.v[0]), "=f"(r.v[1]), "=f"(r.v[2]), "=f"(r.v[3]),
+                       "=f"(r.v[4]), "=f"(r.v[5]), "=f"(r.v[6]), "=f"(r.v[7]) : "l"(p));
+    }
     else if constexpr (KIND == kF32x1) r.v = __ldg(reinterpret_cast<const float*>(p));
     else r.v = __ldg(reinterpret_cast<const uint16_t*>(p));
 }
@@ -482,6 +489,10 @@ __device__ __forceinline__ void zero_raw(Raw<KIND>& r)
 {
     if constexpr (KIND == kF32x4) r.v = make_float4(0.f, 0.f, 0.f, 0.f);
     else if constexpr (KIND == kBF16x8) r.v = make_uint4(0u, 0u, 0u, 0u);
+    else if constexpr (KIND == kF32x8) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) r.v[j] = 0.f;
+    }
     else if constexpr (KIND == kF32x1) r.v = 0.f;
     else r.v = 0;
 }
@@ -490,7 +501,10 @@ template <int KIND>
 __device__ __forceinline__ void unpack(const Raw<KIND>& r, float (&x)[Traits<KIND>::VEC])
 {
     if constexpr (KIND == kF32x4) { x[0] = r.v.x; x[1] = r.v.y; x[2] = r.v.z; x[3] = r.v.w; }
-    else if constexpr (KIND == kBF16x8) {
+    else if constexpr (KIND == kF32x8) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) x[j] = r.v[j];
+    } else if constexpr (KIND == kBF16x8) {
         x[0] = bf16lo(r.v.x); x[1] = bf16hi(r.v.x); x[2] = bf16lo(r.v.y); x[3] = bf16hi(r.v.y);
         x[4] = bf16lo(r.v.z); x[5] = bf16hi(r.v.z); x[6] = bf16lo(r.v.w); x[7] = bf16hi(r.v.w);
     } else if constexpr (KIND == kF32x1) x[0] = r.v;
@@ -499,7 +513,7 @@ __device__ __forceinline__ void unpack(const Raw<KIND>& r, float (&x)[Traits<KIN
 
 template <int KIND> __device__ __forceinline__ constexpr int grad_elem_bytes()
 {
-    return (KIND == kF32x4 || KIND == kF32x1) ? 4 : 2;
+    return (KIND == kF32x4 || KIND == kF32x1 || KIND == kF32x8) ? 4 : 2;
 }
 
 // write this tile's column partial sums (summed over the block's row groups in a fixed order)
@@ -549,7 +563,7 @@ __device__ __forceinline__ void p1_tile(const TensorDev& d, int rb, int cb, cons
                                         Shared& sm)
 {
     constexpr int VEC = Traits<KIND>::VEC;
-    constexpr int U = CAME_P12_U;
+    constexpr int U = (KIND == kF32x8) ? CAME_P12_U / 2 : CAME_P12_U;   // 32 raw registers either way
     const Geo q = make_geo<VEC>(d, rb, cb);
     const int lane = threadIdx.x & 31;
     const long long stride = static_cast<long long>(q.TY) * d.cols * grad_elem_bytes<KIND>();
@@ -602,7 +616,7 @@ __device__ __forceinline__ void p2_tile(const TensorDev& d, int rb, int cb, cons
                                         Shared& sm)
 {
     constexpr int VEC = Traits<KIND>::VEC;
-    constexpr int U = CAME_P12_U;
+    constexpr int U = (KIND == kF32x8) ? CAME_P12_U / 2 : CAME_P12_U;   // 32 raw registers either way
     const Geo q = make_geo<VEC>(d, rb, cb);
     const long long stride = static_cast<long long>(q.TY) * d.cols * grad_elem_bytes<KIND>();
     const char* gp = static_cast<const char*>(d.g) +
@@ -795,7 +809,7 @@ __device__ __forceinline__ void p34_adafactor_tile(const TensorDev& d, int rb, i
                                                    const StepConsts& hc)
 {
     constexpr int VEC = Traits<KIND>::VEC;
-    constexpr int U = CAME_P34_U;
+    constexpr int U = (KIND == kF32x8) ? CAME_P34_U / 2 : CAME_P34_U;   // 24 registers per thread-row there
     const Geo q = make_geo<VEC>(d, rb, cb);
     if (!q.colok) return;
     const long long first = (q.row0 + q.ty) * d.cols + q.col;
@@ -939,6 +953,7 @@ __device__ __forceinline__ void vec_apply_chunk(const TensorDev& d, int chunk, c
     switch (d.kind) {                                                  \
         case kF32x4:  FN<kF32x4>(__VA_ARGS__);  break;                 \
         case kBF16x8: FN<kBF16x8>(__VA_ARGS__); break;                 \
+        case kF32x8:  FN<kF32x8>(__VA_ARGS__);  break;                 \
         case kF32x1:  FN<kF32x1>(__VA_ARGS__);  break;                 \
         default:      FN<kBF16x1>(__VA_ARGS__); break;                 \
     }

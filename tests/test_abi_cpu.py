@@ -91,14 +91,18 @@ def test_plan_covers_matrix_exactly(shape, dt, target):
     assert (p["n_rb"] - 1) * tr < rows <= p["n_rb"] * tr
     assert (p["n_cb"] - 1) * sw < cols <= p["n_cb"] * sw
     assert p["n_rb"] <= 256 or tr >= rows // 256
-    if vec > 1:
-        assert (vec == 8) == (dt == 1)
+    if dt == 1:
+        assert vec in (1, 8)
+    if cols % 8 == 0:
+        assert vec == 8          # 256-bit accesses whenever rows start 32-byte aligned
 
 
 def test_plan_unaligned_bf16_falls_back_to_scalar():
     assert binding.came_plan_tensor(64, 1024, 2, 1, False, 0)["vec"] == 1
     assert binding.came_plan_tensor(64, 1024, 2, 0, False, 0)["vec"] == 4
     assert binding.came_plan_tensor(64, 1022, 2, 0, True, 0)["vec"] == 1
+    assert binding.came_plan_tensor(64, 1024, 2, 0, True, 0)["vec"] == 8
+    assert binding.came_plan_tensor(64, 1028, 2, 0, True, 0)["vec"] == 4
 
 
 def test_plan_rejects_bad_arguments():
