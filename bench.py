@@ -263,9 +263,9 @@ def run_gpu(args):
 TRAFFIC_BYTES = {
     # one-layer capture (profiles/ncu_phase_kernels_llama7b_layer.md) scaled by matrix elements
     ("llama7b", "p4_apply"): 79.33e9,
-    ("llama7b", "p3_momentum_instability"): 66.76e9,
-    ("llama7b_layer", "p4_apply"): 2.3826e9,
-    ("llama7b_layer", "p3_momentum_instability"): 2.0051e9,
+    ("llama7b", "p3_momentum_instability"): 66.75e9,
+    ("llama7b_layer", "p4_apply"): 2.3827e9,
+    ("llama7b_layer", "p3_momentum_instability"): 2.0048e9,
 }
 
 
