@@ -298,3 +298,29 @@ def test_grouped_schedule_and_pipelined_host_step_are_bit_identical(env):
     assert _same(want, b.snapshot())
     for o, p in zip(outs, b.p):
         assert bool((o == p.cpu()).all())
+
+
+def test_two_contexts_on_two_streams_do_not_interfere(env):
+    """Contexts share nothing on the device: stepping two of them concurrently on different
+    streams gives each the result it gets alone."""
+    torch, binding = env
+    alone = []
+    for seed in (21, 22):
+        b = Buffers(torch, binding, W_ODD, seed)
+        ctx = binding.came_create(b.descs)
+        _run_steps(torch, binding, b, ctx, seed, 1, 3)
+        binding.came_destroy(ctx)
+        alone.append(b.snapshot())
+    bufs = [Buffers(torch, binding, W_ODD, seed) for seed in (21, 22)]
+    ctxs = [binding.came_create(b.descs) for b in bufs]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    for step in (1, 2, 3):
+        for b, seed in zip(bufs, (21, 22)):
+            b.set_grads(seed, step)
+        torch.cuda.synchronize()
+        for ctx, st in zip(ctxs, streams):
+            binding.came_step(ctx, binding.make_hparams(step, **HP), None, st.cuda_stream)
+        torch.cuda.synchronize()
+    for ctx in ctxs:
+        binding.came_destroy(ctx)
+    assert _same(alone[0], bufs[0].snapshot()) and _same(alone[1], bufs[1].snapshot())

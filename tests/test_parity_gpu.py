@@ -196,3 +196,44 @@ def test_nan_in_one_tensor_does_not_touch_the_others(env):
     clean, dirty = outs
     for i in (1, 3, 5, 7, 8, 9):                      # everything belonging to tensors 1 and 3
         assert bool((clean[i] == dirty[i]).all())
+
+
+# ---------------------------------------------------------------------------
+# seeded random sweep: shapes, gradient types, tile sizes, hyper-parameters, flags
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("case", range(24))
+def test_random_configurations(env, case):
+    torch, binding, oracle = env
+    rng = np.random.default_rng(1000 + case)
+    def dim():
+        k = rng.integers(0, 4)
+        return int([rng.integers(1, 9), rng.integers(9, 200), rng.integers(200, 1500),
+                    8 * rng.integers(16, 300)][k])
+    ts = []
+    for i in range(int(rng.integers(1, 5))):
+        if rng.random() < 0.25:
+            ts.append(synth.vec(f"v{i}", int(rng.integers(1, 6000))))
+        else:
+            ts.append(synth.mat(f"m{i}", dim(), dim()))
+    dt = synth.BF16 if rng.random() < 0.5 else synth.F32
+    hp = dict(lr=float(10 ** rng.uniform(-5, -2)), beta1=float(rng.choice([0.0, 0.5, 0.9, 0.99])),
+              beta2=float(rng.choice([0.9, 0.999])), beta3=float(rng.choice([0.99, 0.9999])),
+              eps1=float(rng.choice([1e-30, 1e-16, 1e-9])), eps2=float(rng.choice([1e-16, 1e-8])),
+              clip_d=float(rng.choice([0.1, 1.0, 100.0])), weight_decay=float(rng.choice([0.0, 0.01])),
+              grad_scale=float(rng.choice([1.0, 0.125, 3.0])))
+    kind = str(rng.choice(["normal_fixed", "student_t3"]))
+    w = synth.Workload(f"rand{case}", tuple(ts), dt, kind, float(10 ** rng.uniform(-5, -1)), 0.0, (), 4, hp)
+    flags = []
+    for t in ts:
+        f = binding.CAME_T_NO_WEIGHT_DECAY if rng.random() < 0.3 else 0
+        if t.ndim == 1 and rng.random() < 0.3:
+            f |= binding.CAME_T_VEC_NO_CONFIDENCE
+        flags.append(f)
+    binding.came_tune(binding.CAME_TUNE_TILE_ELEMS, int(rng.choice([0, 4096, 16384])))
+    try:
+        res = run_paired(torch, binding, oracle, w, seed=case, steps=4, check_at=(1, 4), flags=flags,
+                         algorithm="adafactor" if rng.random() < 0.2 else "came",
+                         bf16_copy=bool(rng.random() < 0.3))
+    finally:
+        binding.came_tune(binding.CAME_TUNE_TILE_ELEMS, 0)
+    _gate(res)
