@@ -251,11 +251,11 @@ enum {
                                          tensors; per-phase timing is then not reported.  0 = off. */
     CAME_TUNE_HOST_GROUP_BYTES = 2,   /* bytes of gradients + parameters per pipeline stage of
                                          came_step_host (default 1 GiB) */
-    CAME_TUNE_PDL = 3                 /* 1 (default): phase kernels use programmatic dependent
+    CAME_TUNE_PDL = 3,                /* 1 (default): phase kernels use programmatic dependent
                                          launch, so a phase's blocks are scheduled during the
                                          previous phase's tail; 0: plain stream order.  Read at
                                          every step. */
-    , CAME_TUNE_F32_VEC8 = 4          /* 1 (default): fp32 gradients are read 8 per thread with
+    CAME_TUNE_F32_VEC8 = 4            /* 1 (default): fp32 gradients are read 8 per thread with
                                          256-bit loads when rows are 32-byte aligned; 0: 4 per
                                          thread (128-bit) */
 };

@@ -124,3 +124,16 @@ def test_workload_shapes_match_the_named_models():
         assert sum(t.ndim == 2 for t in w.tensors) == nm
         assert sum(t.ndim == 1 for t in w.tensors) == nv
         assert w.numel == numel
+
+
+def test_header_is_plain_c():
+    """The boundary is a C ABI: the header must compile as C99 on its own."""
+    import subprocess, tempfile
+    with tempfile.TemporaryDirectory() as d:
+        src = os.path.join(d, "t.c")
+        with open(src, "w") as f:
+            f.write('#include "came_b200.h"\nint main(void) { came_hparams h; (void)h; return 0; }\n')
+        res = subprocess.run(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror",
+                              "-fsyntax-only", "-I", os.path.join(ROOT, "include"), src],
+                             capture_output=True, text=True)
+        assert res.returncode == 0, res.stderr
