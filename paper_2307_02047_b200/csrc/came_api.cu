@@ -88,7 +88,7 @@ Plan plan_tensor(long long rows, long long cols, int ndim, int dtype, bool align
     p.n_rb = static_cast<int>(ceil_div(rows, tr));
     p.n_seg = p.n_cb * (p.tx / 32);
     p.n_parts = p.n_rb * p.n_cb;
-    p.n_grp = (p.n_rb + came::kColGroup - 1) / came::kColGroup;
+    p.n_grp = (p.n_rb + came::kColGroup - 1) / came::kColGroup;   // <= kColGroup since n_rb <= 256
     return p;
 }
 
@@ -452,6 +452,10 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
         const bool a32 = aligned(x.param, 32) && aligned(x.m, 32) &&
                          (x.grad_dtype == CAME_BF16 || aligned(x.grad, 32));
         Plan p = plan_tensor(x.rows, x.cols, x.ndim, x.grad_dtype, a32, target);
+        if (p.n_grp > came::kColGroup) {      // the two-level column reduction covers 16 x 16 row blocks
+            delete ctx;
+            return fail(nullptr, CAME_ERR_INTERNAL, "tile plan exceeds the column-reduction fan-in");
+        }
         plans[i] = p;
         const long long numel = x.rows * x.cols;
         const long long sg = x.grad_dtype == CAME_BF16 ? 2 : 4;

@@ -122,7 +122,7 @@ __device__ __forceinline__ void load_f(const float* p, float (&x)[VEC])
         asm volatile("ld.global.L1::no_allocate.v4.f32 {%0,%1,%2,%3}, [%4];"
                      : "=f"(x[0]), "=f"(x[1]), "=f"(x[2]), "=f"(x[3]) : "l"(p));
     } else {
-        x[0] = *p;
+        x[0] = __ldcg(p);
     }
 }
 
@@ -311,7 +311,7 @@ __device__ __forceinline__ void finalize_factors(const TensorDev& d, int rb, int
                 float s = 0.f;
 #pragma unroll 8
                 for (int sg = 0; sg < d.n_seg; ++sg) s += __ldcg(d.ws_rowpart + sg * rows + row);
-                const float nv = fmaf(beta, rowfac[row], omb * fmaf(scale, s, add));
+                const float nv = fmaf(beta, __ldcg(rowfac + row), omb * fmaf(scale, s, add));
                 rowfac[row] = nv;
                 d.ws_rowscale[row] = __frsqrt_rn(nv);
                 bs += nv;
@@ -324,7 +324,7 @@ __device__ __forceinline__ void finalize_factors(const TensorDev& d, int rb, int
                 for (int sg = lane; sg < d.n_seg; sg += 32) s += __ldcg(d.ws_rowpart + sg * rows + row);
                 s = warp_sum(s);
                 if (lane == 0) {
-                    const float nv = fmaf(beta, rowfac[row], omb * fmaf(scale, s, add));
+                    const float nv = fmaf(beta, __ldcg(rowfac + row), omb * fmaf(scale, s, add));
                     rowfac[row] = nv;
                     d.ws_rowscale[row] = __frsqrt_rn(nv);
                     bs += nv;
@@ -375,7 +375,7 @@ __device__ __forceinline__ void finalize_factors(const TensorDev& d, int rb, int
                     sum_partial_rows<4>(d.ws_colpart2 + col, cols, d.n_grp, acc);
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        const float nv = fmaf(beta, colfac[col + j], omb * fmaf(scale, acc[j], add));
+                        const float nv = fmaf(beta, __ldcg(colfac + col + j), omb * fmaf(scale, acc[j], add));
                         colfac[col + j] = nv;
                         d.ws_colscale[col + j] = __frsqrt_rn(nv);
                     }
@@ -384,7 +384,7 @@ __device__ __forceinline__ void finalize_factors(const TensorDev& d, int rb, int
                 for (long long col = col0 + tid; col < col1; col += kThreads) {
                     float acc[1];
                     sum_partial_rows<1>(d.ws_colpart2 + col, cols, d.n_grp, acc);
-                    const float nv = fmaf(beta, colfac[col], omb * fmaf(scale, acc[0], add));
+                    const float nv = fmaf(beta, __ldcg(colfac + col), omb * fmaf(scale, acc[0], add));
                     colfac[col] = nv;
                     d.ws_colscale[col] = __frsqrt_rn(nv);
                 }
