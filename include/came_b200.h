@@ -44,7 +44,9 @@
  *   - Every function returns a came_status; nothing is launched when
  *     validation fails.  No exceptions, no abort.  came_last_error gives text.
  *   - came_step enqueues work on the caller's stream and returns without
- *     synchronising.  A context is not re-entrant: one thread at a time.
+ *     synchronising.  A context is not re-entrant: one thread at a time.  The
+ *     context's device must be the calling thread's current device, and the
+ *     stream must belong to it.
  */
 #ifndef CAME_B200_H
 #define CAME_B200_H
