@@ -277,10 +277,10 @@ def run_gpu(args):
 # (workload, kernel).  None until a capture of the current kernel exists.
 TRAFFIC_BYTES = {
     # one-layer capture (profiles/ncu_phase_kernels_llama7b_layer.md) scaled by matrix elements
-    ("llama7b", "p4_apply"): 79.33e9,
-    ("llama7b", "p3_momentum_instability"): 66.75e9,
-    ("llama7b_layer", "p4_apply"): 2.3827e9,
-    ("llama7b_layer", "p3_momentum_instability"): 2.0048e9,
+    ("llama7b", "p4_apply"): 79.37e9,
+    ("llama7b", "p3_momentum_instability"): 66.81e9,
+    ("llama7b_layer", "p4_apply"): 2.3838e9,
+    ("llama7b_layer", "p3_momentum_instability"): 2.0065e9,
 }
 
 
