@@ -376,3 +376,56 @@ def test_optimizer_driver_lists(oracle):
     # first-step magnitude predicted by the closed form (~2.2e-3 per step at the defaults)
     d = np.abs(opt.p[0] - params[0].astype(np.float64))
     assert 1e-3 < d.mean() < 1e-2
+
+
+def test_vector_no_confidence_equals_algorithm1_on_a_column_matrix(oracle):
+    # the alternate vector reading is Algorithm 1 applied to the vector as an N x 1 matrix
+    rng = np.random.default_rng(16)
+    N = 23
+    theta0 = rng.standard_normal(N) * 0.02
+    grads = [rng.standard_normal(N) * 1e-3 for _ in range(4)]
+    hp = dict(HP, weight_decay=0.002, eps1=3e-7)
+    th = theta0.copy(); mo = np.zeros(N); v = np.zeros(N); S = np.zeros(N)
+    TH = theta0.reshape(N, 1).copy(); MO = np.zeros((N, 1)); r = np.zeros(N); c = np.zeros(1)
+    for g in grads:
+        oracle.vector_step(th, g, mo, v, S, oracle.hparams(**hp), no_confidence=True)
+        oracle.adafactor_matrix_step(TH, np.ascontiguousarray(g.reshape(N, 1)), MO, r, c,
+                                     oracle.hparams(**hp))
+    np.testing.assert_allclose(th, TH.ravel(), rtol=1e-11)
+    np.testing.assert_allclose(mo, MO.ravel(), rtol=1e-11)
+    np.testing.assert_allclose(v, r, rtol=1e-12)
+
+
+try:
+    from hypothesis import given, settings, strategies as st
+    _HAVE_HYPOTHESIS = True
+except Exception:                                     # pragma: no cover
+    _HAVE_HYPOTHESIS = False
+
+
+if _HAVE_HYPOTHESIS:
+    @settings(max_examples=25, deadline=None)
+    @given(n=st.integers(1, 12), m=st.integers(1, 12), k=st.integers(-12, 12),
+           seed=st.integers(0, 10_000), steps=st.integers(1, 4))
+    def test_property_invariances_on_random_shapes(n, m, k, seed, steps):
+        """On arbitrary small shapes: power-of-two gradient scaling (eps1 = 0) leaves theta, m,
+        R, C unchanged and scales r, c by 4^k; transposing the problem transposes the result;
+        and the dense-EMA brute force agrees."""
+        from oracle import came_oracle as oracle
+        rng = np.random.default_rng(seed)
+        theta0 = rng.standard_normal((n, m)) * 0.02
+        grads = [_rand_g(rng, n, m) for _ in range(steps)]
+        hp = dict(HP, eps1=0.0, beta3=0.99)
+        base = _run(oracle, theta0, grads, hp)
+        scaled = _run(oracle, theta0, [g * 2.0 ** k for g in grads], hp)
+        for i in (0, 1, 4, 5):
+            np.testing.assert_allclose(scaled[i], base[i], rtol=1e-12)
+        np.testing.assert_allclose(scaled[2], base[2] * 4.0 ** k, rtol=1e-12)
+        np.testing.assert_allclose(scaled[3], base[3] * 4.0 ** k, rtol=1e-12)
+        tr = _run(oracle, np.ascontiguousarray(theta0.T), [np.ascontiguousarray(g.T) for g in grads], hp)
+        np.testing.assert_allclose(tr[0].T, base[0], rtol=1e-9)
+        np.testing.assert_allclose(tr[2], base[3], rtol=1e-10)
+        np.testing.assert_allclose(tr[4], base[5], rtol=1e-9)
+        want = dense_bruteforce(theta0, grads, hp)
+        for a, b in zip(base[:6], want):
+            np.testing.assert_allclose(a, b, rtol=1e-9)
