@@ -45,8 +45,8 @@
  *     validation fails.  No exceptions, no abort.  came_last_error gives text.
  *   - came_step enqueues work on the caller's stream and returns without
  *     synchronising.  A context is not re-entrant: one thread at a time.  The
- *     context's device must be the calling thread's current device, and the
- *     stream must belong to it.
+ *     context's device must be the calling thread's current device (checked:
+ *     CAME_ERR_DEVICE, nothing launched), and the stream must belong to it.
  */
 #ifndef CAME_B200_H
 #define CAME_B200_H
@@ -123,8 +123,12 @@ typedef struct {
     double  beta1;         /* in [0,1)                                     */
     double  beta2;         /* in [0,1)                                     */
     double  beta3;         /* in [0,1)                                     */
-    double  eps1;          /* >= 0, regulariser of g^2                      */
-    double  eps2;          /* >= 0, regulariser of the instability U        */
+    double  eps1;          /* >= 0, regulariser of g^2 (Algorithm 2 uses 1e-30).  With 0 a row
+                              or column of g that is entirely zero gives r_i = 0 (c_j = 0) and
+                              u = 0 / sqrt(0) = NaN there, exactly as Algorithm 2 evaluated
+                              literally does; keep it > 0 unless no such row can occur */
+    double  eps2;          /* >= 0, regulariser of the instability U (1e-16); 0 has the same
+                              consequence for S_t when uhat_t = m_t on a whole row or column */
     double  clip_d;        /* d > 0, RMS clipping threshold (Eq. 1)         */
     double  weight_decay;  /* lambda >= 0 (extension; 0 = the paper)        */
     int64_t step;          /* t >= 1; must be previous + 1 after the first call.  Not used
@@ -159,8 +163,13 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
 /* Algorithm 2, one pass of the loop body over every tensor of the context.
  * `hp`: HOST pointer.  `grads`: HOST array of n DEVICE gradient pointers that
  * replace the ones given at create for this and later steps, or NULL to keep
- * them.  `cuda_stream`: the caller's cudaStream_t (NULL = default stream).
- * Asynchronous; allocates nothing. */
+ * them.  A replacement must be aligned like the pointer it replaces was used: the
+ * launch plan is fixed at create, so where create found an fp32 gradient (with
+ * cols % 8 == 0 and param, m, grad all 32-byte aligned) and planned 256-bit loads,
+ * the replacement must be 32-byte aligned too (came_required_grad_alignment);
+ * everywhere else 16 bytes.  A pointer that is not gives CAME_ERR_ALIGN and
+ * nothing is launched.  `cuda_stream`: the caller's cudaStream_t (NULL = default
+ * stream).  Asynchronous; allocates nothing. */
 came_status came_step(came_ctx* ctx, const came_hparams* hp, const void* const* grads,
                       void* cuda_stream);
 
@@ -210,6 +219,22 @@ came_status came_plan_tensor(int64_t rows, int64_t cols, int32_t ndim, int32_t g
                              int32_t* out_threads_x, int32_t* out_tile_rows, int32_t* out_n_rb,
                              int32_t* out_n_cb);
 
+/* Host-only helpers (no CUDA call).
+ * came_required_grad_alignment: bytes a gradient pointer must be aligned to for a tensor
+ * whose plan reads `vec` elements per thread (came_plan_tensor's out_vec): 32 for fp32
+ * gradients with vec == 8, else 16.
+ * came_device_status: the comparison came_step makes before it launches anything --
+ * CAME_OK when `current_device` (the calling thread's cudaGetDevice) is the device the
+ * context was created on, else CAME_ERR_DEVICE.
+ * came_lr_warmup: the learning rate of step `step` (1-based) under the warm-up the paper's
+ * experiments use (Section 4.1, "Implementation Detail": start from a smaller rate and
+ * increase gradually to eta).  The paper does not give the shape of the ramp; this one is
+ * linear: lr_start + (lr_peak - lr_start) * step / warmup_steps for step < warmup_steps,
+ * lr_peak from then on (and for warmup_steps <= 0).  The value goes into came_hparams.lr. */
+int32_t     came_required_grad_alignment(int32_t grad_dtype, int32_t vec);
+came_status came_device_status(int32_t context_device, int32_t current_device);
+double      came_lr_warmup(double lr_peak, double lr_start, int64_t step, int64_t warmup_steps);
+
 /* Allocation-free factor update (the paper has no counterpart: this exists for callers of
  * this library that are not allowed to allocate device memory).
  *
@@ -240,6 +265,16 @@ came_status came_factor_update_static(const void* grad, int32_t grad_dtype, int6
                                       int64_t cols, float* r, float* c, double beta2,
                                       double eps1, float* out_sqrt_sum_r, int32_t device,
                                       void* cuda_stream);
+
+/* Host-only companion of came_factor_update_static: runs the same argument checks and the
+ * same planning, touches no GPU, launches nothing.  Outputs (HOST, may be NULL): elements per
+ * thread per gradient load (8 = 256-bit loads of fp32, chosen only when `grad` is 32-byte
+ * aligned; 4 = 128-bit; bf16 reads 8 per 128-bit load) and the bytes of the built-in
+ * scratch the call would use.  Returns what the real call would return for these arguments. */
+came_status came_factor_update_static_plan(const void* grad, int32_t grad_dtype, int64_t rows,
+                                           int64_t cols, const float* r, const float* c,
+                                           double beta2, double eps1, int32_t device,
+                                           int32_t* out_vec, int64_t* out_scratch_bytes);
 
 /* Process-wide tuning knobs, read by later came_create calls.  CAME_TUNE_TILE_ELEMS:
  * elements per matrix tile (0 restores the default, which scales with the size

@@ -32,7 +32,9 @@ CAME_TUNE_F32_VEC8 = 4
 
 EXPORTED = ["came_create", "came_step", "came_step_host", "came_destroy", "came_last_error",
             "came_status_string", "came_query", "came_set_profiling", "came_get_phase_ms",
-            "came_phase_name", "came_plan_tensor", "came_tune", "came_factor_update_static"]
+            "came_phase_name", "came_plan_tensor", "came_tune", "came_factor_update_static",
+            "came_factor_update_static_plan", "came_required_grad_alignment",
+            "came_device_status", "came_lr_warmup"]
 
 
 class CameError(RuntimeError):
@@ -96,6 +98,16 @@ def load():
     L.came_factor_update_static.argtypes = [vp, i32, i64, i64, vp, vp, ctypes.c_double,
                                             ctypes.c_double, vp, i32, vp]
     L.came_factor_update_static.restype = i32
+    L.came_factor_update_static_plan.argtypes = [vp, i32, i64, i64, vp, vp, ctypes.c_double,
+                                                 ctypes.c_double, i32, ctypes.POINTER(i32),
+                                                 ctypes.POINTER(i64)]
+    L.came_factor_update_static_plan.restype = i32
+    L.came_required_grad_alignment.argtypes = [i32, i32]
+    L.came_required_grad_alignment.restype = i32
+    L.came_device_status.argtypes = [i32, i32]
+    L.came_device_status.restype = i32
+    L.came_lr_warmup.argtypes = [ctypes.c_double, ctypes.c_double, i64, i64]
+    L.came_lr_warmup.restype = ctypes.c_double
     _lib = L
     return L
 
@@ -196,6 +208,28 @@ def came_factor_update_static(grad: int, grad_dtype: int, rows: int, cols: int, 
     _check(load().came_factor_update_static(grad, grad_dtype, rows, cols, r, c, float(beta2),
                                             float(eps1), out_sqrt_sum_r, device,
                                             ctypes.c_void_p(stream)))
+
+
+def came_factor_update_static_plan(grad: int, grad_dtype: int, rows: int, cols: int, r: int, c: int,
+                                   beta2: float = 0.999, eps1: float = 1e-30, device: int = 0) -> dict:
+    """Host-only: what came_factor_update_static would plan for these arguments (no GPU work)."""
+    vec, nbytes = ctypes.c_int32(), ctypes.c_int64()
+    _check(load().came_factor_update_static_plan(grad, grad_dtype, rows, cols, r, c, float(beta2),
+                                                 float(eps1), device, ctypes.byref(vec),
+                                                 ctypes.byref(nbytes)))
+    return {"vec": int(vec.value), "scratch_bytes": int(nbytes.value)}
+
+
+def came_required_grad_alignment(grad_dtype: int, vec: int) -> int:
+    return int(load().came_required_grad_alignment(grad_dtype, vec))
+
+
+def came_device_status(context_device: int, current_device: int) -> int:
+    return int(load().came_device_status(context_device, current_device))
+
+
+def came_lr_warmup(lr_peak: float, lr_start: float, step: int, warmup_steps: int) -> float:
+    return float(load().came_lr_warmup(lr_peak, lr_start, step, warmup_steps))
 
 
 def make_hparams(step: int, **kw) -> came_hparams:

@@ -144,6 +144,14 @@ came_status cuda_fail(came_ctx* ctx, cudaError_t e, const char* what)
 
 bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
+// Byte alignment a gradient pointer must have for a plan that reads `vec` elements per
+// thread per load: 8 fp32 elements are one 256-bit load (32 bytes); every other plan reads at
+// most 128 bits at a time, and 16 bytes is the contract for all tensor pointers.
+size_t grad_alignment_for(int grad_dtype, int vec)
+{
+    return (grad_dtype == CAME_F32 && vec == 8) ? 32 : 16;
+}
+
 came_status validate_tensor(const came_tensor& t, int i, bool adafactor, std::string& msg)
 {
     char buf[160];
@@ -343,9 +351,42 @@ std::vector<Group> make_groups(const came_ctx* ctx, long long limit, F bytes_of)
     return out;
 }
 
+// A step launched with another device current would run on that GPU with this context's
+// pointers.  The comparison itself is came_device_status, so it can be exercised without a GPU.
+came_status check_current_device(came_ctx* ctx)
+{
+    int cur = -1;
+    const cudaError_t e = cudaGetDevice(&cur);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaGetDevice");
+    if (came_device_status(ctx->device, cur) != CAME_OK) {
+        char buf[120];
+        std::snprintf(buf, sizeof buf, "the context lives on device %d but device %d is current",
+                      ctx->device, cur);
+        return fail(ctx, CAME_ERR_DEVICE, buf);
+    }
+    return CAME_OK;
+}
+
 }  // namespace
 
 extern "C" {
+
+came_status came_device_status(int32_t context_device, int32_t current_device)
+{
+    return (context_device >= 0 && context_device == current_device) ? CAME_OK : CAME_ERR_DEVICE;
+}
+
+int32_t came_required_grad_alignment(int32_t grad_dtype, int32_t vec)
+{
+    return static_cast<int32_t>(grad_alignment_for(grad_dtype, vec));
+}
+
+double came_lr_warmup(double lr_peak, double lr_start, int64_t step, int64_t warmup_steps)
+{
+    if (warmup_steps <= 0 || step >= warmup_steps) return lr_peak;
+    if (step < 0) step = 0;
+    return lr_start + (lr_peak - lr_start) * (static_cast<double>(step) / static_cast<double>(warmup_steps));
+}
 
 const char* came_status_string(came_status s)
 {
@@ -587,12 +628,21 @@ came_status came_step(came_ctx* ctx, const came_hparams* hp, const void* const* 
     std::string msg;
     came_status s = validate_hparams(*hp, ctx->last_step, msg);
     if (s != CAME_OK) return fail(ctx, s, msg);
+    s = check_current_device(ctx);
+    if (s != CAME_OK) return s;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     if (grads) {
         bool changed = false;
         for (int i = 0; i < ctx->n; ++i) {
             if (!grads[i]) return fail(ctx, CAME_ERR_NULL, "a gradient pointer is NULL");
-            if (!aligned(grads[i], 16)) return fail(ctx, CAME_ERR_ALIGN, "gradient pointer not 16-byte aligned");
+            // the tile plan (and with it the width of the loads) was fixed at create
+            const size_t need = grad_alignment_for(ctx->tensors[i].grad_dtype, ctx->host_table[i].vec);
+            if (!aligned(grads[i], need)) {
+                char buf[120];
+                std::snprintf(buf, sizeof buf, "tensor %d: replacement gradient pointer not %zu-byte aligned",
+                              i, need);
+                return fail(ctx, CAME_ERR_ALIGN, buf);
+            }
             changed |= (grads[i] != ctx->host_table[i].g);
         }
         if (changed) {
@@ -614,6 +664,8 @@ came_status came_step_host(came_ctx* ctx, const came_hparams* hp, const void* co
     if (s != CAME_OK) return fail(ctx, s, msg);
     for (int i = 0; i < ctx->n; ++i)
         if (!host_grads[i]) return fail(ctx, CAME_ERR_NULL, "a host gradient pointer is NULL");
+    s = check_current_device(ctx);
+    if (s != CAME_OK) return s;
     cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
     const StepConsts hc = make_consts(*hp);
     cudaError_t e;
@@ -776,10 +828,22 @@ k_p1_reduce_g2_single(const TensorDev d, StepConsts hc)
 
 }  // namespace
 
-extern "C" came_status came_factor_update_static(const void* grad, int32_t grad_dtype, int64_t rows,
-                                                 int64_t cols, float* r, float* c, double beta2,
-                                                 double eps1, float* out_sqrt_sum_r, int32_t device,
-                                                 void* cuda_stream)
+namespace {
+
+struct StaticLayout {
+    Plan p;
+    size_t need = 0;
+    size_t colpart = 0, colpart2 = 0, rowpart = 0, blocksum = 0, rowscale = 0, colscale = 0, cnt = 0,
+           scal = 0;
+};
+
+// Host-only: validates the arguments of came_factor_update_static and lays its partial sums
+// out in the built-in scratch array.  The tile grows (fewer, taller tiles) until they fit.
+// The width of the gradient loads follows the pointer actually passed: 256-bit loads of fp32
+// gradients only when it is 32-byte aligned, else 128-bit.
+came_status plan_static(const void* grad, int32_t grad_dtype, int64_t rows, int64_t cols,
+                        const float* r, const float* c, double beta2, double eps1, int32_t device,
+                        StaticLayout& L)
 {
     if (!grad || !r || !c) return fail(nullptr, CAME_ERR_NULL, "grad, r and c are required");
     if (rows < 1 || cols < 1 || rows > (1ll << 40) / cols)
@@ -793,35 +857,65 @@ extern "C" came_status came_factor_update_static(const void* grad, int32_t grad_
     if (device < 0 || device >= kMaxDevices)
         return fail(nullptr, CAME_ERR_DEVICE, "device ordinal out of range");
 
-    // Lay the scratch out; grow the tile until the partial sums fit (fewer, taller tiles).
-    Plan p;
-    size_t need = 0;
-    struct { size_t colpart, colpart2, rowpart, blocksum, rowscale, colscale, cnt, scal; } off{};
+    const bool a32 = grad_dtype == CAME_BF16 || aligned(grad, 32);
     for (long long target = 32768; ; target *= 2) {
-        p = plan_tensor(rows, cols, 2, grad_dtype, true, target);
+        Plan& p = L.p;
+        p = plan_tensor(rows, cols, 2, grad_dtype, a32, target);
         size_t ws = 0;
         auto take = [&](size_t bytes) { const size_t o = ws; ws += (bytes + 255) / 256 * 256; return o; };
-        off.cnt = take(sizeof(unsigned) * p.counters());
-        off.scal = take(sizeof(float) * 4);
-        off.blocksum = take(sizeof(float) * p.n_rb);
-        off.colpart = take(sizeof(float) * static_cast<size_t>(p.n_rb) * cols);
-        off.colpart2 = take(sizeof(float) * static_cast<size_t>(p.n_grp) * cols);
-        off.rowpart = take(sizeof(float) * static_cast<size_t>(p.n_seg) * rows);
-        off.rowscale = take(sizeof(float) * static_cast<size_t>(rows));
-        off.colscale = take(sizeof(float) * static_cast<size_t>(cols));
-        need = ws;
-        if (need <= CAME_STATIC_SCRATCH_BYTES || p.n_rb == 1 || target >= (1ll << 40)) break;
+        L.cnt = take(sizeof(unsigned) * p.counters());
+        L.scal = take(sizeof(float) * 4);
+        L.blocksum = take(sizeof(float) * p.n_rb);
+        L.colpart = take(sizeof(float) * static_cast<size_t>(p.n_rb) * cols);
+        L.colpart2 = take(sizeof(float) * static_cast<size_t>(p.n_grp) * cols);
+        L.rowpart = take(sizeof(float) * static_cast<size_t>(p.n_seg) * rows);
+        L.rowscale = take(sizeof(float) * static_cast<size_t>(rows));
+        L.colscale = take(sizeof(float) * static_cast<size_t>(cols));
+        L.need = ws;
+        if (L.need <= CAME_STATIC_SCRATCH_BYTES || p.n_rb == 1 || target >= (1ll << 40)) break;
     }
-    if (need > CAME_STATIC_SCRATCH_BYTES) {
+    if (L.need > CAME_STATIC_SCRATCH_BYTES) {
         char buf[200];
         std::snprintf(buf, sizeof buf,
                       "matrix %lld x %lld needs %zu bytes of partial sums; the built-in scratch holds %u",
-                      static_cast<long long>(rows), static_cast<long long>(cols), need,
+                      static_cast<long long>(rows), static_cast<long long>(cols), L.need,
                       static_cast<unsigned>(CAME_STATIC_SCRATCH_BYTES));
         return fail(nullptr, CAME_ERR_UNSUPPORTED, buf);
     }
-    if (static_cast<long long>(p.n_rb) * p.n_cb > (1ll << 30))
+    if (static_cast<long long>(L.p.n_rb) * L.p.n_cb > (1ll << 30))
         return fail(nullptr, CAME_ERR_SHAPE, "too many tiles");
+    if (grad_alignment_for(grad_dtype, L.p.vec) > 16 && !aligned(grad, 32))
+        return fail(nullptr, CAME_ERR_INTERNAL, "plan wider than the gradient pointer's alignment");
+    return CAME_OK;
+}
+
+}  // namespace
+
+extern "C" came_status came_factor_update_static_plan(const void* grad, int32_t grad_dtype,
+                                                      int64_t rows, int64_t cols, const float* r,
+                                                      const float* c, double beta2, double eps1,
+                                                      int32_t device, int32_t* out_vec,
+                                                      int64_t* out_scratch_bytes)
+{
+    StaticLayout L;
+    const came_status s = plan_static(grad, grad_dtype, rows, cols, r, c, beta2, eps1, device, L);
+    if (s != CAME_OK) return s;
+    if (out_vec) *out_vec = L.p.vec;
+    if (out_scratch_bytes) *out_scratch_bytes = static_cast<int64_t>(L.need);
+    return CAME_OK;
+}
+
+extern "C" came_status came_factor_update_static(const void* grad, int32_t grad_dtype, int64_t rows,
+                                                 int64_t cols, float* r, float* c, double beta2,
+                                                 double eps1, float* out_sqrt_sum_r, int32_t device,
+                                                 void* cuda_stream)
+{
+    StaticLayout off;
+    const came_status st = plan_static(grad, grad_dtype, rows, cols, r, c, beta2, eps1, device, off);
+    if (st != CAME_OK) return st;
+    if (out_sqrt_sum_r && !aligned(out_sqrt_sum_r, 4))
+        return fail(nullptr, CAME_ERR_ALIGN, "out_sqrt_sum_r not 4-byte aligned");
+    const Plan& p = off.p;
 
     cudaError_t e = cudaSetDevice(device);
     if (e != cudaSuccess) { cudaGetLastError(); return fail(nullptr, CAME_ERR_DEVICE, "cudaSetDevice failed"); }

@@ -137,3 +137,61 @@ def test_header_is_plain_c():
                               "-fsyntax-only", "-I", os.path.join(ROOT, "include"), src],
                              capture_output=True, text=True)
         assert res.returncode == 0, res.stderr
+
+
+# ---------------------------------------------------------------------------
+# alignment and device checks that must hold before anything is launched
+# ---------------------------------------------------------------------------
+def test_static_plan_follows_the_gradient_pointer_alignment():
+    """The allocation-free entry point plans 256-bit loads of fp32 gradients only for a
+    32-byte aligned pointer; a pointer at 16 mod 32 (a view into a flat buffer) gets 128-bit
+    loads, never a wider access than its alignment allows."""
+    base, r, c = 0x7f0000000000, 0x7f0000100000, 0x7f0000200000
+    F32, BF16 = binding.CAME_F32, binding.CAME_BF16
+    plan = binding.came_factor_update_static_plan
+    assert plan(base, F32, 512, 1024, r, c)["vec"] == 8
+    assert plan(base + 16, F32, 512, 1024, r, c)["vec"] == 4
+    assert plan(base + 16, F32, 512, 1028, r, c)["vec"] == 4        # cols % 8 != 0
+    assert plan(base, F32, 512, 1028, r, c)["vec"] == 4
+    assert plan(base + 16, F32, 512, 1030, r, c)["vec"] == 1
+    assert plan(base + 16, BF16, 512, 1024, r, c)["vec"] == 8       # one 128-bit load of 8 bf16
+    for off in (4, 8, 2):
+        with pytest.raises(binding.CameError) as e:
+            plan(base + off, F32, 512, 1024, r, c)
+        assert e.value.status == 4
+    with pytest.raises(binding.CameError) as e:
+        plan(base, F32, 3_000_000, 4, r, c)
+    assert e.value.status == 11
+    assert plan(base, F32, 4096, 4096, r, c)["scratch_bytes"] <= binding.CAME_STATIC_SCRATCH_BYTES
+    for a in range(0, 64, 16):
+        v = plan(base + a, F32, 64, 4096, r, c)["vec"]
+        assert (base + a) % binding.came_required_grad_alignment(F32, v) == 0
+
+
+def test_required_gradient_alignment():
+    assert binding.came_required_grad_alignment(binding.CAME_F32, 8) == 32
+    assert binding.came_required_grad_alignment(binding.CAME_F32, 4) == 16
+    assert binding.came_required_grad_alignment(binding.CAME_F32, 1) == 16
+    assert binding.came_required_grad_alignment(binding.CAME_BF16, 8) == 16
+    assert binding.came_required_grad_alignment(binding.CAME_BF16, 1) == 16
+
+
+def test_device_status_comparison():
+    assert binding.came_device_status(0, 0) == 0
+    assert binding.came_device_status(3, 3) == 0
+    assert binding.came_device_status(0, 1) == 7
+    assert binding.came_device_status(1, 0) == 7
+    assert binding.came_device_status(-1, -1) == 7
+
+
+def test_lr_warmup_is_a_linear_ramp_to_the_peak():
+    f = binding.came_lr_warmup
+    assert f(2e-4, 0.0, 1, 10) == pytest.approx(2e-5, rel=1e-15)
+    assert f(2e-4, 0.0, 5, 10) == pytest.approx(1e-4, rel=1e-15)
+    assert f(2e-4, 0.0, 10, 10) == 2e-4
+    assert f(2e-4, 0.0, 11, 10) == 2e-4
+    assert f(2e-4, 1e-5, 0, 10) == 1e-5
+    assert f(2e-4, 1e-5, 4, 8) == pytest.approx(1e-5 + 0.5 * (2e-4 - 1e-5), rel=1e-15)
+    assert f(6e-4, 0.0, 3, 0) == 6e-4
+    vals = [f(3e-4, 0.0, t, 100) for t in range(0, 120)]
+    assert all(b >= a for a, b in zip(vals, vals[1:])) and max(vals) == 3e-4

@@ -324,3 +324,63 @@ def test_two_contexts_on_two_streams_do_not_interfere(env):
     for ctx in ctxs:
         binding.came_destroy(ctx)
     assert _same(alone[0], bufs[0].snapshot()) and _same(alone[1], bufs[1].snapshot())
+
+
+def test_replacement_gradient_must_match_the_planned_load_width(env):
+    """The launch plan is fixed at create.  A tensor planned for 256-bit fp32 gradient loads
+    rejects a replacement pointer at 16 mod 32 before anything is launched; a tensor planned
+    for 128-bit loads accepts it and gives the result of the aligned buffer."""
+    torch, binding = env
+    w = synth.Workload("align", (synth.mat("a", 64, 1024), synth.mat("b", 64, 1028)), synth.F32,
+                       "normal_fixed", 1e-3, 0.0, (), 2, HP)
+    assert binding.came_plan_tensor(64, 1024, 2, 0, True)["vec"] == 8
+    assert binding.came_plan_tensor(64, 1028, 2, 0, True)["vec"] == 4
+    stream = torch.cuda.current_stream().cuda_stream
+    ref = Buffers(torch, binding, w, 17)
+    ctx = binding.came_create(ref.descs)
+    _run_steps(torch, binding, ref, ctx, 17, 1, 2)
+    binding.came_destroy(ctx)
+
+    buf = Buffers(torch, binding, w, 17)
+    for x in buf.g:
+        assert x.data_ptr() % 32 == 0
+    ctx = binding.came_create(buf.descs)
+    _run_steps(torch, binding, buf, ctx, 17, 1, 1)
+    before = buf.snapshot()
+    buf.set_grads(17, 2)
+    shifted = []
+    for g in buf.g:                       # the same values, 16 bytes into a larger buffer
+        big = torch.zeros(g.numel() + 16, dtype=torch.float32, device="cuda:0")
+        off = ((16 - big.data_ptr() % 32) % 32) // 4
+        view = big[off:off + g.numel()]
+        view.copy_(g)
+        assert view.data_ptr() % 32 == 16
+        shifted.append((big, view))
+    with pytest.raises(binding.CameError) as e:
+        binding.came_step(ctx, binding.make_hparams(2, **HP),
+                          [shifted[0][1].data_ptr(), buf.g[1].data_ptr()], stream)
+    assert e.value.status == 4 and "32-byte" in str(e.value)
+    assert _same(before, buf.snapshot())
+    assert binding.came_query(ctx, binding.CAME_Q_LAST_STEP) == 1
+    binding.came_step(ctx, binding.make_hparams(2, **HP),
+                      [buf.g[0].data_ptr(), shifted[1][1].data_ptr()], stream)
+    torch.cuda.synchronize()
+    binding.came_destroy(ctx)
+    buf.check_guards()
+    assert _same(ref.snapshot(), buf.snapshot())
+
+
+def test_step_with_another_device_current_is_refused(env):
+    torch, binding = env
+    if torch.cuda.device_count() < 2:
+        pytest.skip("needs two GPUs; the comparison itself is covered by the CPU test of came_device_status")
+    buf = Buffers(torch, binding, synth.workload("toy"), 19)
+    ctx = binding.came_create(buf.descs, device=0)
+    buf.set_grads(19, 1)
+    before = buf.snapshot()
+    with torch.cuda.device(1):
+        with pytest.raises(binding.CameError) as e:
+            binding.came_step(ctx, binding.make_hparams(1, **HP), None, 0)
+    assert e.value.status == 7
+    assert _same(before, buf.snapshot())
+    binding.came_destroy(ctx)

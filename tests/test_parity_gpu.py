@@ -4,7 +4,7 @@ import numpy as np
 import pytest
 
 from paper_2307_02047_b200 import synth
-from tests.parity_util import TOL_STEP1, TOL_STEP10, run_paired
+from tests.parity_util import TOL_STEP1, TOL_STEP10, gate, run_paired
 
 pytestmark = pytest.mark.gpu
 
@@ -19,10 +19,7 @@ def env(oracle):
 
 
 def _gate(res):
-    for step, worst in res.items():
-        tol = TOL_STEP1 if step == 1 else TOL_STEP10
-        for name, e in worst.items():
-            assert e <= tol, f"step {step}: {name} error {e:.3e} > {tol:.0e}  ({worst})"
+    gate(res)
 
 
 def test_toy_config_ten_steps(env):
@@ -64,7 +61,9 @@ def test_vectors(env, n):
 def test_flags_weight_decay_and_no_confidence(env):
     torch, binding, oracle = env
     ts = (synth.mat("w0", 130, 264), synth.mat("w1", 64, 128), synth.vec("b0", 300), synth.vec("b1", 300))
-    hp = dict(synth.PAPER_HPARAMS, weight_decay=0.01)
+    # lr * lambda * |theta| is 2e-4 of the first update here: a dropped decay term, or a
+    # dropped opt-out flag, moves the cumulative update by 20 times the step-1 gate
+    hp = dict(synth.PAPER_HPARAMS, lr=1e-3, weight_decay=0.1)
     w = synth.Workload("flags", ts, synth.BF16, "student_t3", 1e-3, 0.0, (), 10, hp)
     flags = [0, binding.CAME_T_NO_WEIGHT_DECAY, binding.CAME_T_VEC_NO_CONFIDENCE,
              binding.CAME_T_NO_WEIGHT_DECAY]
