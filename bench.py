@@ -187,13 +187,14 @@ def run_gpu(args):
             sampler.start()
             time.sleep(0.3)
         barrier()
-        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        ev0.record()
-        for _ in range(args.steps):
+        marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
+        marks[0].record()
+        for k in range(args.steps):
             opt.step(**hp)
-        ev1.record()
+            marks[k + 1].record()
         barrier()
-        ms = ev0.elapsed_time(ev1)
+        ms = marks[0].elapsed_time(marks[-1])
+        ms_median = _median([marks[k].elapsed_time(marks[k + 1]) for k in range(args.steps)])
         clocks = sampler.stop() if rank == 0 else {}
         phase_ms = binding.came_get_phase_ms(opt.ctx)
         phase_names = [binding.came_phase_name(opt.ctx, i) for i in range(len(phase_ms))]
@@ -220,6 +221,7 @@ def run_gpu(args):
     barrier()
     ms_plain = max_over_ranks(ev2.elapsed_time(ev3), world, device) / args.steps
     ms = max_over_ranks(ms, world, device)
+    ms_median = max_over_ranks(ms_median, world, device)
     ms_per_step = ms / args.steps
     value = job_value(world, numel, ms_per_step)
 
@@ -238,7 +240,8 @@ def run_gpu(args):
         ach = pb[dom] / (matrix_phases[dom] * 1e-3) / 1e9
         roofline = {"bound": "hbm", "kernel": dom, "achieved": round(ach, 1), "peak": peak,
                     "peak_kind": peak_kind, "unit": "GB/s", "frac": round(ach / peak, 4),
-                    "traffic": TRAFFIC_BYTES.get((args.workload, dom)),
+                    "traffic": traffic_bytes(args.workload, dom),
+                    "kernel_source_hash": kernel_source_hash(),
                     "algorithmic_bytes_per_launch": pb[dom],
                     "per_phase": {n: {"ms": round(m, 4), "GB/s": round(pb[n] / (m * 1e-3) / 1e9, 1)}
                                   for n, m in matrix_phases.items()}}
@@ -246,6 +249,7 @@ def run_gpu(args):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
+        "ms_per_step_median": ms_median,
         "ms_per_step_without_phase_events": ms_plain, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": args.workload, "algorithm": args.algorithm, "params": numel,
@@ -263,9 +267,16 @@ def run_gpu(args):
         "clocks": clocks, "e2e": e2e, "gpu_launches": launches * args.steps,
         "roofline": roofline,
     }
+    opt.close()
+    del opt, params, grads
+    torch.cuda.empty_cache()
+    if world == 1 and not args.no_configs and args.workload == "llama7b":
+        # the other configurations, after the headline run has freed its memory: each is a
+        # few milliseconds per step, so they cost nothing next to the headline's set-up
+        line["configs"] = {name: time_config(torch, binding, name, device, peak, peak_kind)
+                           for name in EXTRA_CONFIGS}
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         line["cpu_baseline"] = cpu_baseline(budget_s=25.0, steps=1, warmup=0)
-    opt.close()
     if world > 1:
         dist.barrier()
         dist.destroy_process_group()
@@ -273,8 +284,82 @@ def run_gpu(args):
         print(json.dumps(line), flush=True)
 
 
+EXTRA_CONFIGS = ("bert_base", "bert_large", "gpt2_medium", "mat:16384x16384", "mat:128256x4096")
+SCHEDULE_NAMES = {0: "one grid per phase", 1: "pipelined persistent grid"}
+
+
+def _median(xs):
+    xs = sorted(xs)
+    n = len(xs)
+    return xs[n // 2] if n % 2 else 0.5 * (xs[n // 2 - 1] + xs[n // 2])
+
+
+def time_config(torch, binding, name, device, peak, peak_kind, steps=20, warmup=5):
+    """Median step time of one further workload (device-resident, CUDA events around every
+    step), then the same steps again with the per-phase events on for the per-kernel figures."""
+    w = synth.workload(name)
+    hp = dict(w.hparams)
+    params, grads = alloc_device_workload(torch, w, device)
+    opt = binding.CameOptimizer(params, grads, device=device.index or 0)
+    stream_bytes = opt.query(binding.CAME_Q_STREAM_BYTES)
+    comp_bytes = opt.query(binding.CAME_Q_COMPULSORY_BYTES)
+    numel = opt.query(binding.CAME_Q_NUMEL)
+    for _ in range(warmup):
+        opt.step(**hp)
+    torch.cuda.synchronize()
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    marks[0].record()
+    for k in range(steps):
+        opt.step(**hp)
+        marks[k + 1].record()
+    torch.cuda.synchronize()
+    per_step = [marks[k].elapsed_time(marks[k + 1]) for k in range(steps)]
+    ms = _median(per_step)
+    binding.came_set_profiling(opt.ctx, True)
+    for _ in range(steps):
+        opt.step(**hp)
+    torch.cuda.synchronize()
+    per_phase = {}
+    try:
+        phase_ms = binding.came_get_phase_ms(opt.ctx)
+        pb = phase_bytes(w)
+        for i, m in enumerate(phase_ms):
+            n = binding.came_phase_name(opt.ctx, i)
+            if n in pb and m > 0:
+                g = pb[n] / (m * 1e-3) / 1e9
+                per_phase[n] = {"ms": round(m, 4), "GB/s": round(g, 1),
+                                "frac_of_%s" % peak_kind: round(g / peak, 3)}
+    except binding.CameError:
+        per_phase = None
+    binding.came_set_profiling(opt.ctx, False)
+    sg = 2 if w.grad_dtype == synth.BF16 else 4
+    gbs = stream_bytes / (ms * 1e-3) / 1e9
+    sched = opt.query(binding.CAME_Q_SCHEDULE) if hasattr(binding, "CAME_Q_SCHEDULE") else 0
+    out = {"params": numel, "ms_per_step_median": round(ms, 4),
+           "ms_per_step_min": round(min(per_step), 4), "steps": steps, "warmup": warmup,
+           "params_per_s": numel / (ms * 1e-3),
+           "stream_bytes_per_step": stream_bytes, "compulsory_bytes_per_step": comp_bytes,
+           "effective_GBps": round(gbs, 1),
+           "frac_of_nominal_8TBps": round(gbs / NOMINAL_HBM_GBS, 4),
+           "frac_of_%s_%.1f" % (peak_kind, peak): round(gbs / peak, 4),
+           "tiles": opt.query(binding.CAME_Q_NUM_TILES),
+           "schedule": SCHEDULE_NAMES.get(sched, "?"),
+           "per_phase": per_phase,
+           "l2": "p, m and g of the set are %.2f GB against a 126 MB L2 (largest tensor's g + m: %.0f MB): "
+                 "inputs larger than L2, no flush between steps"
+                 % (sum(t.numel for t in w.tensors) * (8 + sg) / 1e9,
+                    max(t.numel for t in w.tensors) * (4 + sg) / 1e6)}
+    opt.close()
+    del opt, params, grads
+    torch.cuda.empty_cache()
+    return out
+
+
 # ncu-measured DRAM bytes per launch of the dominant kernel (read + write), keyed by
-# (workload, kernel).  None until a capture of the current kernel exists.
+# (workload, kernel).  The figures belong to one build of the kernels: TRAFFIC_KERNEL_HASH is
+# kernel_source_hash() of the sources they were captured on, and traffic_bytes() answers None
+# (the JSON line then says "traffic": null) as soon as the sources differ.
+TRAFFIC_KERNEL_HASH = "0000000000000000"
 TRAFFIC_BYTES = {
     # one-layer capture (profiles/ncu_phase_kernels_llama7b_layer.md) scaled by matrix elements
     ("llama7b", "p4_apply"): 79.37e9,
@@ -282,6 +367,23 @@ TRAFFIC_BYTES = {
     ("llama7b_layer", "p4_apply"): 2.3838e9,
     ("llama7b_layer", "p3_momentum_instability"): 2.0065e9,
 }
+
+
+def kernel_source_hash() -> str:
+    import hashlib
+    h = hashlib.sha256()
+    base = os.path.join(ROOT, "paper_2307_02047_b200", "csrc")
+    for name in sorted(os.listdir(base)):
+        if name.endswith((".cu", ".cuh")):
+            with open(os.path.join(base, name), "rb") as f:
+                h.update(name.encode() + b"\0" + f.read())
+    return h.hexdigest()[:16]
+
+
+def traffic_bytes(workload: str, kernel: str):
+    if kernel_source_hash() != TRAFFIC_KERNEL_HASH:
+        return None
+    return TRAFFIC_BYTES.get((workload, kernel))
 
 
 def host_mem_available() -> int:
@@ -392,12 +494,35 @@ def time_oracle(sample: synth.Workload, steps: int, warmup: int):
     return dt, came_oracle.threads()
 
 
+def oracle_single_thread() -> dict:
+    """The same oracle on ONE host thread (a child process with OMP_NUM_THREADS=1, so the
+    oracle itself is untouched), on one 4096 x 4096 matrix of the LLaMA-7B-shaped set."""
+    code = ("import sys, time, json; sys.path.insert(0, %r)\n"
+            "from paper_2307_02047_b200 import synth\n"
+            "from oracle import came_oracle\n"
+            "w = synth.Workload('one', (synth.mat('wq', 4096, 4096),), synth.BF16, 'normal_fixed', 1e-3,"
+            " 0.0, (), 1, dict(synth.PAPER_HPARAMS))\n"
+            "o = came_oracle.OracleOptimizer(synth.make_params(w, 1))\n"
+            "g = [synth.widen(x) for x in synth.make_grads(w, 1, 1)]\n"
+            "t0 = time.perf_counter(); o.step(g, **w.hparams); dt = time.perf_counter() - t0\n"
+            "print(json.dumps({'dt': dt, 'numel': w.numel, 'threads': came_oracle.threads()}))\n" % ROOT)
+    try:
+        res = subprocess.run([sys.executable, "-c", code], capture_output=True, text=True, timeout=300,
+                             env=dict(os.environ, OMP_NUM_THREADS="1"))
+        r = json.loads(res.stdout.strip().splitlines()[-1])
+        return {"value": r["numel"] / r["dt"], "unit": UNIT, "cores": r["threads"],
+                "sample": "one 4096x4096 matrix (16.8 M parameters), 1 step, %.2f s" % r["dt"]}
+    except Exception as e:                       # reported, never fatal for the GPU line
+        return {"value": None, "error": str(e)[:200]}
+
+
 def cpu_baseline(budget_s: float, steps: int, warmup: int) -> dict:
     sample, desc = _oracle_sample(budget_s, steps + warmup)
     dt, threads = time_oracle(sample, steps, warmup)
     return {"value": sample.numel / dt, "unit": UNIT, "cores": threads, "kind": "oracle",
             "sample": desc + f"; {steps} step(s), {dt:.2f} s per step; throughput per parameter is "
-                             "size-independent (tensors are independent)"}
+                             "size-independent (tensors are independent)",
+            "single_thread": oracle_single_thread()}
 
 
 def run_reference(args):
@@ -431,6 +556,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")
+    ap.add_argument("--no-configs", action="store_true",
+                    help="skip the further configurations timed after the headline workload")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)
