@@ -149,7 +149,13 @@ enum {
     CAME_Q_LAUNCHES_PER_STEP = 6,/* kernels one came_step enqueues                               */
     CAME_Q_LAST_STEP = 7,        /* last step accepted (0 before the first)                      */
     CAME_Q_NUM_PHASES = 8,       /* entries came_get_phase_ms reports                            */
-    CAME_Q_MATRIX_NUMEL = 9      /* elements that live in matrices (the four-phase path)         */
+    CAME_Q_MATRIX_NUMEL = 9,     /* elements that live in matrices (the four-phase path)         */
+    CAME_Q_SCHEDULE = 10,        /* 0 = one grid per phase, 1 = pipelined persistent grid        */
+    CAME_Q_PIPE_GROUPS = 11,     /* pipelined schedule: tensor groups (pipeline stages)          */
+    CAME_Q_PIPE_GRID = 12,       /* pipelined schedule: blocks of the persistent grid            */
+    CAME_Q_DEVICE_ERROR = 13     /* pipelined schedule: 0, or the error word a step left on the
+                                    device (low 8 bits: 1 = a bounded wait ran out; upper bits:
+                                    the work item that gave up).  SYNCHRONISES the device. */
 };
 
 /* Algorithm 2, set-up.  Validates `t[0..n)` (HOST array of descriptors holding
@@ -198,6 +204,22 @@ const char* came_status_string(came_status s);
 
 /* Facts about the context; `what` is a CAME_Q_* selector, *out a HOST int64. */
 came_status came_query(const came_ctx* ctx, int32_t what, int64_t* out);
+
+/* The pipelined schedule waits, inside its one grid, for per-tensor "phase done" flags; each
+ * wait is bounded (CAME_TUNE_PIPE_WAIT_NS, 2 s by default).  If a wait ever runs out, the grid
+ * records an error word and returns; later steps of the context then do nothing (they leave
+ * every buffer untouched) until the caller, having seen CAME_Q_DEVICE_ERROR != 0, calls
+ * came_clear_device_error, which re-zeroes the context's counters, flags and control block
+ * on `cuda_stream`.  State tensors may hold a partly applied step at that point: restore them
+ * from the caller's last checkpoint.  Harmless on a context that uses the other schedule. */
+came_status came_clear_device_error(came_ctx* ctx, void* cuda_stream);
+
+/* Self-test of that bounded wait, without a context: one thread waits, with the limit given
+ * (1 us .. 1 s), for a flag that nothing sets.  Outputs (HOST): whether the wait reported a
+ * time-out (1 expected), the error word it left (1 expected), and the device time the kernel
+ * took.  Allocates and frees 16 bytes of device memory; synchronises. */
+came_status came_selftest_wait_timeout(int32_t device, int64_t limit_ns, int32_t* out_timed_out,
+                                       int32_t* out_error_word, float* out_elapsed_ms);
 
 /* Per-phase device timing.  When enabled, came_step records CUDA events on the
  * caller's stream between its kernels (no synchronisation); switching it on
@@ -292,9 +314,24 @@ enum {
                                          launch, so a phase's blocks are scheduled during the
                                          previous phase's tail; 0: plain stream order.  Read at
                                          every step. */
-    CAME_TUNE_F32_VEC8 = 4            /* 1 (default): fp32 gradients are read 8 per thread with
+    CAME_TUNE_F32_VEC8 = 4,           /* 1 (default): fp32 gradients are read 8 per thread with
                                          256-bit loads when rows are 32-byte aligned; 0: 4 per
                                          thread (128-bit) */
+    CAME_TUNE_SCHEDULE = 5,           /* schedule of contexts created afterwards: 0 = chosen from
+                                         the tensor sizes, 1 = one grid per phase (four launches),
+                                         2 = pipelined: the whole step is ONE persistent grid whose
+                                         blocks draw (tensor, tile, phase) items in an order that
+                                         sends L2-sized groups of tensors through the phases one
+                                         pipeline stage apart, so a group's gradient is read from
+                                         HBM once and its momentum is still in the L2 when the last
+                                         phase reads it.  Same arithmetic, same results. */
+    CAME_TUNE_PIPE_TILE_ELEMS = 6,    /* pipelined schedule: elements per tile (0 = default 8192) */
+    CAME_TUNE_PIPE_GROUP_BYTES = 7,   /* pipelined schedule: bytes of gradient + momentum per
+                                         tensor group (0 = default 20 MiB) */
+    CAME_TUNE_PIPE_WAIT_NS = 8,       /* pipelined schedule: limit of every wait for a flag, in
+                                         nanoseconds (0 = default 2 s) */
+    CAME_TUNE_PIPE_ORDER = 9          /* pipelined schedule: 0 = groups one stage apart (default),
+                                         1 = each group's phases back to back */
 };
 came_status came_tune(int32_t key, int64_t value);
 

@@ -23,18 +23,26 @@ CAME_CREATE_KEEP_STATE = 1
 CAME_CREATE_ADAFACTOR = 2
 (CAME_Q_NUMEL, CAME_Q_STATE_BYTES, CAME_Q_STREAM_BYTES, CAME_Q_COMPULSORY_BYTES,
  CAME_Q_WORKSPACE_BYTES, CAME_Q_NUM_TILES, CAME_Q_LAUNCHES_PER_STEP, CAME_Q_LAST_STEP,
- CAME_Q_NUM_PHASES, CAME_Q_MATRIX_NUMEL) = range(10)
+ CAME_Q_NUM_PHASES, CAME_Q_MATRIX_NUMEL, CAME_Q_SCHEDULE, CAME_Q_PIPE_GROUPS, CAME_Q_PIPE_GRID,
+ CAME_Q_DEVICE_ERROR) = range(14)
 CAME_TUNE_TILE_ELEMS = 0
 CAME_TUNE_SCHED_GROUP_BYTES = 1
 CAME_TUNE_HOST_GROUP_BYTES = 2
 CAME_TUNE_PDL = 3
 CAME_TUNE_F32_VEC8 = 4
+CAME_TUNE_SCHEDULE = 5
+CAME_TUNE_PIPE_TILE_ELEMS = 6
+CAME_TUNE_PIPE_GROUP_BYTES = 7
+CAME_TUNE_PIPE_WAIT_NS = 8
+CAME_TUNE_PIPE_ORDER = 9
+CAME_SCHEDULE_AUTO, CAME_SCHEDULE_PHASE_GRIDS, CAME_SCHEDULE_PIPELINED = 0, 1, 2
 
 EXPORTED = ["came_create", "came_step", "came_step_host", "came_destroy", "came_last_error",
             "came_status_string", "came_query", "came_set_profiling", "came_get_phase_ms",
             "came_phase_name", "came_plan_tensor", "came_tune", "came_factor_update_static",
             "came_factor_update_static_plan", "came_required_grad_alignment",
-            "came_device_status", "came_lr_warmup"]
+            "came_device_status", "came_lr_warmup", "came_clear_device_error",
+            "came_selftest_wait_timeout"]
 
 
 class CameError(RuntimeError):
@@ -108,6 +116,11 @@ def load():
     L.came_device_status.restype = i32
     L.came_lr_warmup.argtypes = [ctypes.c_double, ctypes.c_double, i64, i64]
     L.came_lr_warmup.restype = ctypes.c_double
+    L.came_clear_device_error.argtypes = [vp, vp]
+    L.came_clear_device_error.restype = i32
+    L.came_selftest_wait_timeout.argtypes = [i32, i64, ctypes.POINTER(i32), ctypes.POINTER(i32),
+                                             ctypes.POINTER(ctypes.c_float)]
+    L.came_selftest_wait_timeout.restype = i32
     _lib = L
     return L
 
@@ -230,6 +243,17 @@ def came_device_status(context_device: int, current_device: int) -> int:
 
 def came_lr_warmup(lr_peak: float, lr_start: float, step: int, warmup_steps: int) -> float:
     return float(load().came_lr_warmup(lr_peak, lr_start, step, warmup_steps))
+
+
+def came_clear_device_error(ctx, stream: int = 0) -> None:
+    _check(load().came_clear_device_error(ctx, ctypes.c_void_p(stream)), ctx)
+
+
+def came_selftest_wait_timeout(device: int = 0, limit_ns: int = 1_000_000) -> dict:
+    a, b, ms = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_float()
+    _check(load().came_selftest_wait_timeout(device, limit_ns, ctypes.byref(a), ctypes.byref(b),
+                                             ctypes.byref(ms)))
+    return {"timed_out": int(a.value), "error_word": int(b.value), "elapsed_ms": float(ms.value)}
 
 
 def make_hparams(step: int, **kw) -> came_hparams:

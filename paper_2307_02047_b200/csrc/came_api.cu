@@ -29,6 +29,18 @@ bool g_use_pdl = true;                 // came_tune(CAME_TUNE_PDL)
 long long g_sched_group_bytes = 0;     // came_tune(CAME_TUNE_SCHED_GROUP_BYTES); 0 = one group
 long long g_host_group_bytes = 1ll << 30;   // came_tune(CAME_TUNE_HOST_GROUP_BYTES)
 
+int g_schedule = 0;                    // came_tune(CAME_TUNE_SCHEDULE): 0 auto, 1 phase grids, 2 pipelined
+long long g_pipe_tile_elems = 0;       // came_tune(CAME_TUNE_PIPE_TILE_ELEMS); 0 = default
+long long g_pipe_group_bytes = 0;      // came_tune(CAME_TUNE_PIPE_GROUP_BYTES); 0 = default
+long long g_pipe_wait_ns = 0;          // came_tune(CAME_TUNE_PIPE_WAIT_NS); 0 = default (2 s)
+long long g_pipe_order = 0;            // came_tune(CAME_TUNE_PIPE_ORDER)
+constexpr long long kPipeTileElemsDefault = 8192;
+constexpr long long kPipeGroupBytesDefault = 20ll << 20;
+constexpr long long kPipeWaitNsDefault = 2000000000ll;
+constexpr bool kPipeAutoEnabled = false;              // auto never picks the pipelined grid yet
+constexpr long long kPipeAutoTensorBytes = 40ll << 20;
+constexpr long long kPipeAutoMinTenths = 5;
+
 bool g_f32_vec8 = true;                // came_tune(CAME_TUNE_F32_VEC8)
 inline bool g_f32_vec8_ok(bool bf) { return bf || g_f32_vec8; }
 
@@ -119,6 +131,13 @@ struct came_ctx {
     size_t ws_bytes = 0, table_bytes = 0;
     long long numel = 0, matrix_numel = 0, state_bytes = 0, stream_bytes = 0, comp_bytes = 0;
     long long last_step = 0;
+    bool pipelined = false;                    // one persistent grid per step instead of one grid per phase
+    came::Item* d_items = nullptr;             // pipelined schedule: work items in ticket order
+    int n_items = 0;
+    came::PipeSync* d_sync = nullptr;
+    int pipe_grid = 0;                         // blocks of the persistent grid
+    int pipe_groups = 0;
+    unsigned long long pipe_wait_ns = 0;
     bool adafactor = false;                    // Algorithm 1 instead of Algorithm 2
     bool profiling = false;
     std::vector<cudaEvent_t> prof_ev;          // [kProfSlots][kMaxPhases + 1], made on demand
@@ -231,6 +250,8 @@ void free_ctx(came_ctx* ctx)
     cudaFree(ctx->d_table);
     cudaFree(ctx->d_tiles);
     cudaFree(ctx->d_ws);
+    cudaFree(ctx->d_items);
+    cudaFree(ctx->d_sync);
     for (int k = 0; k < 2; ++k) {
         if (ctx->pinned_table[k]) cudaFreeHost(ctx->pinned_table[k]);
         if (ctx->pinned_free[k]) cudaEventDestroy(ctx->pinned_free[k]);
@@ -315,7 +336,17 @@ int launch_range(const came_ctx* ctx, const StepConsts& hc, cudaStream_t stream,
 came_status launch_step(came_ctx* ctx, const came_hparams* hp, cudaStream_t stream)
 {
     const StepConsts hc = make_consts(*hp);
-    if (ctx->sched_groups.empty()) {
+    if (ctx->pipelined) {
+        const bool prof = ctx->profiling && !ctx->prof_ev.empty();
+        cudaEvent_t* ev = prof ? &ctx->prof_ev[(ctx->prof_count % kProfSlots) * (kMaxPhases + 1)] : nullptr;
+        if (ev) cudaEventRecord(ev[0], stream);
+        came::k_step_pipelined<<<ctx->pipe_grid, came::kThreads, 0, stream>>>(
+            ctx->d_table, ctx->d_items, ctx->n_items, ctx->d_sync, hc, ctx->adafactor ? 1 : 0,
+            ctx->pipe_wait_ns);
+        if (ev) cudaEventRecord(ev[1], stream);
+        ctx->n_intervals = 1;
+        if (prof) ++ctx->prof_count;
+    } else if (ctx->sched_groups.empty()) {
         const bool prof = ctx->profiling && !ctx->prof_ev.empty();
         cudaEvent_t* ev = prof ? &ctx->prof_ev[(ctx->prof_count % kProfSlots) * (kMaxPhases + 1)] : nullptr;
         const Group all{0, ctx->n, 0, ctx->n_tiles};
@@ -349,6 +380,63 @@ std::vector<Group> make_groups(const came_ctx* ctx, long long limit, F bytes_of)
         }
     }
     return out;
+}
+
+// Which schedule a new context gets.  came_tune(CAME_TUNE_SCHEDULE) forces one; otherwise the
+// pipelined grid is taken when most of the matrix elements sit in tensors whose gradient and
+// momentum together are small enough for several of them to share the L2.
+bool choose_pipelined(const came_tensor* t, int n)
+{
+    if (g_schedule == 1) return false;
+    if (g_schedule == 2) return true;
+    long long small = 0, all = 0;
+    for (int i = 0; i < n; ++i) {
+        if (t[i].ndim != 2) continue;
+        const long long numel = t[i].rows * t[i].cols;
+        const long long resident = numel * (4 + (t[i].grad_dtype == CAME_BF16 ? 2 : 4));
+        all += numel;
+        if (resident <= kPipeAutoTensorBytes) small += numel;
+    }
+    return kPipeAutoEnabled && all > 0 && small * 10 >= all * kPipeAutoMinTenths;
+}
+
+// Ticket order of the pipelined schedule.  Consecutive tensors form a group until the group's
+// gradients and momenta reach the group size; stage s then holds, oldest first, P4 of group
+// s-3, P3 of group s-2, P2 of group s-1 and P1 of group s.  Every item therefore comes after
+// all items of the phase it depends on (they sit in the stage before), with two other
+// sub-phases in between, which is what keeps the waits short.
+std::vector<came::Item> build_pipeline_items(came_ctx* ctx, const std::vector<Tile>& tiles)
+{
+    const long long group_bytes = g_pipe_group_bytes > 0 ? g_pipe_group_bytes : kPipeGroupBytesDefault;
+    auto resident = [](const came_tensor& x) {
+        return x.rows * x.cols * (4ll + (x.grad_dtype == CAME_BF16 ? 2 : 4)); };
+    const std::vector<Group> groups = make_groups(ctx, group_bytes, resident);
+    ctx->pipe_groups = static_cast<int>(groups.size());
+    const int phases = ctx->adafactor ? 3 : 4;
+    const int ng = static_cast<int>(groups.size());
+    std::vector<came::Item> items;
+    items.reserve(tiles.size() * phases);
+    auto emit = [&](const Group& g, int phase) {
+        for (int k = g.tile0; k < g.tile1; ++k) {
+            const Tile& tl = tiles[k];
+            const bool vec = ctx->tensors[tl.tensor].ndim == 1;
+            if (vec && phase != 0 && phase != 2) continue;     // vectors: two halves only
+            items.push_back(came::Item{tl.tensor, tl.rb, tl.cb, phase});
+        }
+    };
+    if (g_pipe_order == 1) {
+        // no skew: every group runs its phases back to back (dependent items are adjacent,
+        // so the waits are real; kept for tests and measurements)
+        for (int s = 0; s < ng; ++s)
+            for (int ph = 0; ph < phases; ++ph) emit(groups[s], ph);
+        return items;
+    }
+    for (int s = 0; s < ng + phases - 1; ++s)
+        for (int ph = phases - 1; ph >= 0; --ph) {
+            const int grp = s - ph;
+            if (grp >= 0 && grp < ng) emit(groups[grp], ph);
+        }
+    return items;
 }
 
 // A step launched with another device current would run on that GPU with this context's
@@ -421,6 +509,11 @@ came_status came_tune(int32_t key, int64_t value)
         case CAME_TUNE_PDL: g_use_pdl = value != 0; break;
         case CAME_TUNE_F32_VEC8: g_f32_vec8 = value != 0; break;
         case CAME_TUNE_HOST_GROUP_BYTES: g_host_group_bytes = value > 0 ? value : (1ll << 30); break;
+        case CAME_TUNE_SCHEDULE: if (value > 2) return CAME_ERR_UNSUPPORTED; g_schedule = static_cast<int>(value); break;
+        case CAME_TUNE_PIPE_TILE_ELEMS: g_pipe_tile_elems = value; break;
+        case CAME_TUNE_PIPE_GROUP_BYTES: g_pipe_group_bytes = value; break;
+        case CAME_TUNE_PIPE_WAIT_NS: g_pipe_wait_ns = value; break;
+        case CAME_TUNE_PIPE_ORDER: if (value > 1) return CAME_ERR_UNSUPPORTED; g_pipe_order = value; break;
         default: return CAME_ERR_UNSUPPORTED;
     }
     return CAME_OK;
@@ -475,7 +568,10 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
     long long matrix_numel = 0;
     for (int i = 0; i < n; ++i)
         if (t[i].ndim == 2) matrix_numel += t[i].rows * t[i].cols;
+    ctx->pipelined = choose_pipelined(t, n);
     long long target = g_tile_elems_override;
+    if (target <= 0 && ctx->pipelined)
+        target = g_pipe_tile_elems > 0 ? g_pipe_tile_elems : kPipeTileElemsDefault;
     if (target <= 0) {
         // aim for a few thousand tiles in all; between 4 Ki and 256 Ki elements per tile
         target = 4096;
@@ -486,7 +582,7 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
     std::vector<Tile> tiles;
     size_t ws = 0;
     auto take = [&](size_t bytes) { const size_t off = ws; ws += (bytes + 255) / 256 * 256; return off; };
-    struct Off { size_t colpart, colpart2, rowpart, blocksum, usq, cnt, scal, rowscale, colscale; };
+    struct Off { size_t colpart, colpart2, rowpart, blocksum, usq, cnt, scal, rowscale, colscale, done; };
     std::vector<Off> offs(n);
     for (int i = 0; i < n; ++i) {
         const came_tensor& x = t[i];
@@ -533,6 +629,7 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
         offs[i].usq = take(sizeof(float) * p.n_parts);
         offs[i].cnt = take(sizeof(unsigned) * p.counters());
         offs[i].scal = take(sizeof(float) * 4);
+        offs[i].done = take(sizeof(unsigned) * 4);
         ctx->tile_begin[i + 1] = static_cast<int>(tiles.size());
         if (tiles.size() > (1u << 30)) {
             delete ctx;
@@ -554,6 +651,27 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
         CAME_TRY(cudaMalloc(&ctx->d_tiles, sizeof(Tile) * tiles.size()), "cudaMalloc(tiles)");
         CAME_TRY(cudaMemcpy(ctx->d_tiles, tiles.data(), sizeof(Tile) * tiles.size(),
                             cudaMemcpyHostToDevice), "cudaMemcpy(tiles)");
+    }
+    if (ctx->pipelined) {
+        if (tiles.size() > (1u << 28)) {
+            free_ctx(ctx);
+            return fail(nullptr, CAME_ERR_SHAPE, "too many tiles for the pipelined schedule");
+        }
+        const std::vector<came::Item> items = build_pipeline_items(ctx, tiles);
+        ctx->n_items = static_cast<int>(items.size());
+        CAME_TRY(cudaMalloc(&ctx->d_items, sizeof(came::Item) * std::max<size_t>(items.size(), 1)),
+                 "cudaMalloc(items)");
+        CAME_TRY(cudaMemcpy(ctx->d_items, items.data(), sizeof(came::Item) * items.size(),
+                            cudaMemcpyHostToDevice), "cudaMemcpy(items)");
+        CAME_TRY(cudaMalloc(&ctx->d_sync, sizeof(came::PipeSync)), "cudaMalloc(sync)");
+        CAME_TRY(cudaMemset(ctx->d_sync, 0, sizeof(came::PipeSync)), "cudaMemset(sync)");
+        int sms = 0, per_sm = 0;
+        CAME_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device), "cudaDeviceGetAttribute");
+        CAME_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, came::k_step_pipelined,
+                                                               came::kThreads, 0), "occupancy query");
+        ctx->pipe_grid = std::max(1, std::min(ctx->n_items, sms * std::max(per_sm, 1)));
+        ctx->pipe_wait_ns = static_cast<unsigned long long>(g_pipe_wait_ns > 0 ? g_pipe_wait_ns
+                                                                                : kPipeWaitNsDefault);
     }
     for (int k = 0; k < 2; ++k) {
         CAME_TRY(cudaMallocHost(&ctx->pinned_table[k], ctx->table_bytes), "cudaMallocHost(table)");
@@ -595,6 +713,7 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
         d.ws_colscale = reinterpret_cast<float*>(ctx->d_ws + offs[i].colscale);
         d.cnt = reinterpret_cast<unsigned*>(ctx->d_ws + offs[i].cnt);
         d.scal = reinterpret_cast<float*>(ctx->d_ws + offs[i].scal);
+        d.done = reinterpret_cast<unsigned*>(ctx->d_ws + offs[i].done);
         d.kind = p.kind; d.vec = p.vec;
         int lg = 0; while ((1 << lg) < p.tx) ++lg;
         d.tx_log2 = lg; d.tr = p.tr; d.n_rb = p.n_rb; d.n_cb = p.n_cb; d.n_seg = p.n_seg;
@@ -729,17 +848,85 @@ came_status came_query(const came_ctx* ctx, int32_t what, int64_t* out)
         case CAME_Q_STREAM_BYTES: *out = ctx->stream_bytes; break;
         case CAME_Q_COMPULSORY_BYTES: *out = ctx->comp_bytes; break;
         case CAME_Q_WORKSPACE_BYTES:
-            *out = static_cast<int64_t>(ctx->ws_bytes + ctx->table_bytes + sizeof(Tile) * ctx->n_tiles);
+            *out = static_cast<int64_t>(ctx->ws_bytes + ctx->table_bytes + sizeof(Tile) * ctx->n_tiles +
+                                        sizeof(came::Item) * ctx->n_items +
+                                        (ctx->d_sync ? sizeof(came::PipeSync) : 0));
             break;
         case CAME_Q_NUM_TILES: *out = ctx->n_tiles; break;
         case CAME_Q_LAUNCHES_PER_STEP:
-            *out = ctx->adafactor ? 3 : 4; break;
+            *out = ctx->pipelined ? 1 : (ctx->adafactor ? 3 : 4); break;
         case CAME_Q_LAST_STEP: *out = ctx->last_step; break;
         case CAME_Q_NUM_PHASES:
-            *out = ctx->adafactor ? 3 : 4; break;
+            *out = ctx->pipelined ? 1 : (ctx->adafactor ? 3 : 4); break;
         case CAME_Q_MATRIX_NUMEL: *out = ctx->matrix_numel; break;
+        case CAME_Q_SCHEDULE: *out = ctx->pipelined ? 1 : 0; break;
+        case CAME_Q_PIPE_GROUPS: *out = ctx->pipe_groups; break;
+        case CAME_Q_PIPE_GRID: *out = ctx->pipe_grid; break;
+        case CAME_Q_DEVICE_ERROR: {
+            *out = 0;
+            if (ctx->pipelined) {
+                came::PipeSync h;
+                const cudaError_t e = cudaMemcpy(&h, ctx->d_sync, sizeof h, cudaMemcpyDeviceToHost);
+                if (e != cudaSuccess) return CAME_ERR_CUDA;
+                *out = h.error ? (static_cast<int64_t>(h.error) | (static_cast<int64_t>(h.err_item) << 8)) : 0;
+            }
+            break;
+        }
         default: return CAME_ERR_UNSUPPORTED;
     }
+    return CAME_OK;
+}
+
+came_status came_clear_device_error(came_ctx* ctx, void* cuda_stream)
+{
+    if (!ctx) return CAME_ERR_NULL;
+    const came_status s = check_current_device(ctx);
+    if (s != CAME_OK) return s;
+    cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+    // arrival counters, flags and partial sums all start from zero again
+    cudaError_t e = cudaMemsetAsync(ctx->d_ws, 0, std::max<size_t>(ctx->ws_bytes, 256), stream);
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaMemsetAsync(workspace)");
+    if (ctx->d_sync) {
+        e = cudaMemsetAsync(ctx->d_sync, 0, sizeof(came::PipeSync), stream);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaMemsetAsync(sync)");
+    }
+    return CAME_OK;
+}
+
+came_status came_selftest_wait_timeout(int32_t device, int64_t limit_ns, int32_t* out_timed_out,
+                                       int32_t* out_error_word, float* out_elapsed_ms)
+{
+    if (!out_timed_out || !out_error_word || !out_elapsed_ms)
+        return fail(nullptr, CAME_ERR_NULL, "output pointer is NULL");
+    if (limit_ns < 1000 || limit_ns > 1000000000ll)
+        return fail(nullptr, CAME_ERR_UNSUPPORTED, "limit_ns must lie in [1 us, 1 s]");
+    cudaError_t e = cudaSetDevice(device);
+    if (e != cudaSuccess) { cudaGetLastError(); return fail(nullptr, CAME_ERR_DEVICE, "cudaSetDevice failed"); }
+    unsigned* d = nullptr;
+    cudaEvent_t a = nullptr, b = nullptr;
+    came_status st = CAME_OK;
+    unsigned h[4] = {0, 0, 0, 0};
+    float ms = 0.f;
+    do {
+        if ((e = cudaMalloc(&d, sizeof h)) != cudaSuccess) break;
+        if ((e = cudaMemset(d, 0, sizeof h)) != cudaSuccess) break;
+        if ((e = cudaEventCreate(&a)) != cudaSuccess) break;
+        if ((e = cudaEventCreate(&b)) != cudaSuccess) break;
+        cudaEventRecord(a, 0);
+        came::k_wait_probe<<<1, 32>>>(d, static_cast<unsigned long long>(limit_ns));
+        cudaEventRecord(b, 0);
+        if ((e = cudaGetLastError()) != cudaSuccess) break;
+        if ((e = cudaMemcpy(h, d, sizeof h, cudaMemcpyDeviceToHost)) != cudaSuccess) break;
+        if ((e = cudaEventElapsedTime(&ms, a, b)) != cudaSuccess) break;
+    } while (false);
+    if (e != cudaSuccess) st = cuda_fail(nullptr, e, "wait self-test");
+    if (a) cudaEventDestroy(a);
+    if (b) cudaEventDestroy(b);
+    cudaFree(d);
+    if (st != CAME_OK) return st;
+    *out_timed_out = static_cast<int32_t>(h[3]);
+    *out_error_word = static_cast<int32_t>(h[1]);
+    *out_elapsed_ms = ms;
     return CAME_OK;
 }
 
@@ -787,6 +974,7 @@ came_status came_get_phase_ms(came_ctx* ctx, float* out_ms, int32_t cap, int32_t
 const char* came_phase_name(const came_ctx* ctx, int32_t phase)
 {
     if (!ctx || phase < 0) return "";
+    if (ctx->pipelined) return phase == 0 ? "step_pipelined" : "";
     // phases are reported in launch order
     const bool ada = ctx->adafactor;
     const bool has[kMaxPhases] = {true, true, !ada, !ada, ada};

@@ -15,8 +15,20 @@
 // Reductions are deterministic: every tile writes its partial sums to a
 // workspace and the LAST tile to arrive (per row block; per group of 16 row
 // blocks of a column strip, then per strip; per tensor -- counted with atomics)
-// adds them in a fixed order.  No thread ever waits on another block, so there
-// is no spin anywhere in this file.
+// adds them in a fixed order.  In the one-grid-per-phase schedule no thread ever
+// waits on another block.
+//
+// Second schedule, k_step_pipelined: ONE persistent grid runs the whole step.  Its blocks
+// draw tickets, in order, from a list of (tensor, tile, phase) items that the host has
+// arranged so that groups of tensors small enough for the L2 move through P1..P4 one
+// pipeline stage apart: a group's gradient is read from HBM once (P1) and from the L2 in P2
+// and P3, and its momentum written by P3 is still in the L2 when P4 reads it.  An item that
+// needs a tensor-wide result (r,c / kappa / R,C) of an earlier phase waits for that tensor's
+// "phase done" flag.  Every flag an item waits for is set by items with LOWER ticket numbers,
+// and a ticket is only ever held by a block that is running, so the lowest unfinished ticket
+// can always proceed: the waits end without any assumption about how many blocks are
+// resident.  Each wait is nevertheless bounded (time and iteration limit): when it runs out
+// the block records an error word and every block leaves the grid.
 #pragma once
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -69,6 +81,8 @@ struct TensorDev {
     unsigned*    cnt;          // [n_rb] row-block arrivals, [n_cb] finished groups per strip,
                                // [1] finished, [1] usq, [n_grp*n_cb] arrivals per (group, strip)
     float*       scal;         // [0] sqrt(sum r)  [1] kappa  [2] sqrt(sum R)
+    unsigned*    done;         // pipelined schedule: [0] r,c final  [1] kappa final  [2] R,C final,
+                               // each holding the number of the last step that finished it
     uint16_t*    p_bf16;       // optional bf16 copy of the updated parameters (NULL = none)
     int          kind;
     int          vec;          // elements per thread per load
@@ -82,6 +96,22 @@ struct TensorDev {
 };
 
 struct Tile { int tensor, rb, cb; };   // vectors: rb = chunk of kVecChunk elements, cb = 0
+
+// One unit of work of the pipelined schedule: a tile (or vector chunk) in one phase.
+// phase 0 = P1 (vectors: second moment and kappa), 1 = P2, 2 = P3 (vectors: apply;
+// Algorithm 1: the fused momentum + apply pass), 3 = P4.
+struct Item { int tensor, rb, cb, phase; };
+
+// Device-resident control block of the pipelined schedule (one per context).
+struct PipeSync {
+    unsigned ticket;      // next item to hand out; reset by the last block to leave
+    unsigned exited;      // blocks that have left the current grid
+    unsigned epoch;       // number of steps completed; a step publishes flags equal to epoch + 1
+    unsigned error;       // 0 = fine; kPipeErr* once a wait has run out (sticky until cleared)
+    unsigned err_item;    // ticket whose wait ran out
+    unsigned pad_[3];
+};
+constexpr unsigned kPipeErrWaitTimeout = 1u;
 
 struct StepConsts {
     float beta1, omb1, b1sq;
@@ -268,6 +298,55 @@ __device__ __forceinline__ void sum_partial_rows(const float* __restrict__ p, lo
 }
 
 // ---------------------------------------------------------------------------
+// "phase done" flags of the pipelined schedule.  The writer has made its results visible
+// (fence, block barrier, counted arrival) before it publishes; the reader acquires the flag
+// in one thread and the block barrier that follows orders every thread's later loads after it.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ void publish_flag(unsigned* flag, unsigned epoch)
+{
+    __threadfence();
+    asm volatile("st.release.gpu.global.u32 [%0], %1;" :: "l"(flag), "r"(epoch) : "memory");
+}
+
+__device__ __forceinline__ unsigned load_acquire(const unsigned* p)
+{
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+__device__ __forceinline__ unsigned long long global_timer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Called by ONE thread.  Polls until *flag == epoch, another block has reported an error, or
+// the limit runs out (limit_ns of wall time, and as a backstop limit_ns / 8 + 4096 polls, each
+// of which takes well over 8 ns).  Returns true when the flag arrived.  On a timeout the
+// error word is set (first reporter wins) and false is returned; the caller must then leave.
+__device__ __forceinline__ bool wait_for_flag(const unsigned* flag, unsigned epoch,
+                                              unsigned* error_word, unsigned* err_item,
+                                              unsigned item, unsigned long long limit_ns)
+{
+    if (load_acquire(flag) == epoch) return true;
+    const unsigned long long t0 = global_timer_ns();
+    const unsigned long long max_polls = limit_ns / 8ull + 4096ull;
+    unsigned ns = 32;
+    for (unsigned long long it = 0; it < max_polls; ++it) {
+        if (load_acquire(flag) == epoch) return true;
+        if (load_acquire(error_word) != 0u) return false;
+        if (global_timer_ns() - t0 > limit_ns) break;
+        __nanosleep(ns);
+        if (ns < 1024) ns <<= 1;
+    }
+    if (atomicCAS(error_word, 0u, kPipeErrWaitTimeout) == 0u) *err_item = item;
+    __threadfence();
+    return false;
+}
+
+// ---------------------------------------------------------------------------
 // Last-arriver finalisation of one factored EMA (Algorithm 2: r_t, c_t from g^2
 // with beta2/eps1; R_t, C_t from U_t with beta3/eps2):
 //   row[i] = beta row[i] + (1-beta) (scale * sum_j X[i][j] + cols * eps)
@@ -280,7 +359,8 @@ __device__ __forceinline__ void finalize_factors(const TensorDev& d, int rb, int
                                                  float omb, float eps, float scale,
                                                  float* __restrict__ rowfac,
                                                  float* __restrict__ colfac,
-                                                 float* __restrict__ sqrt_sum, Shared& sm)
+                                                 float* __restrict__ sqrt_sum, Shared& sm,
+                                                 unsigned* done_flag = nullptr, unsigned epoch = 0u)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int grp = rb / kColGroup;
@@ -406,14 +486,19 @@ __device__ __forceinline__ void finalize_factors(const TensorDev& d, int rb, int
         double s = 0.0;
         for (int k = tid; k < d.n_rb; k += kThreads) s += static_cast<double>(__ldcg(d.ws_blocksum + k));
         s = block_sum(s, sm);
-        if (tid == 0) { *sqrt_sum = static_cast<float>(sqrt(s)); d.cnt[d.n_rb + d.n_cb] = 0u; }
+        if (tid == 0) {
+            *sqrt_sum = static_cast<float>(sqrt(s));
+            d.cnt[d.n_rb + d.n_cb] = 0u;
+            if (done_flag) publish_flag(done_flag, epoch);   // everything of this factor pair is final
+        }
     }
 }
 
 // Eq. 1: the last part to arrive adds all partial sums of u^2 in a fixed order
 // and stores kappa = 1 / max(1, RMS(u)/d), RMS over all rows*cols components.
 __device__ __forceinline__ void finalize_kappa(const TensorDev& d, int part, float partial,
-                                               double clip_d, Shared& sm)
+                                               double clip_d, Shared& sm,
+                                               unsigned* done_flag = nullptr, unsigned epoch = 0u)
 {
     const int tid = threadIdx.x;
     if (tid == 0) d.ws_usq[part] = partial;
@@ -433,6 +518,7 @@ __device__ __forceinline__ void finalize_kappa(const TensorDev& d, int part, flo
         const double rms = sqrt(s / (static_cast<double>(d.rows) * static_cast<double>(d.cols)));
         d.scal[1] = static_cast<float>(1.0 / fmax(1.0, rms / clip_d));
         d.cnt[d.n_rb + d.n_cb + 1] = 0u;
+        if (done_flag) publish_flag(done_flag, epoch);
     }
 }
 
@@ -560,7 +646,7 @@ __device__ __forceinline__ void store_row_partials(float (&rs)[U], float* __rest
 // ---------------------------------------------------------------------------
 template <int KIND>
 __device__ __forceinline__ void p1_tile(const TensorDev& d, int rb, int cb, const StepConsts& hc,
-                                        Shared& sm)
+                                        Shared& sm, unsigned* done_flag = nullptr, unsigned epoch = 0u)
 {
     constexpr int VEC = Traits<KIND>::VEC;
     constexpr int U = (KIND == kF32x8) ? CAME_P12_U / 2 : CAME_P12_U;   // 32 raw registers either way
@@ -605,7 +691,8 @@ __device__ __forceinline__ void p1_tile(const TensorDev& d, int rb, int cb, cons
         store_row_partials<U>(rs, rowpart_seg, rbase, q.TY, q.row1, lane);
     }
     write_col_partials<VEC>(d, q, rb, cacc, sm);
-    finalize_factors(d, rb, cb, hc.beta2, hc.omb2, hc.eps1, hc.gscale2, d.r, d.c, d.scal + 0, sm);
+    finalize_factors(d, rb, cb, hc.beta2, hc.omb2, hc.eps1, hc.gscale2, d.r, d.c, d.scal + 0, sm,
+                     done_flag, epoch);
 }
 
 // ---------------------------------------------------------------------------
@@ -613,7 +700,7 @@ __device__ __forceinline__ void p1_tile(const TensorDev& d, int rb, int cb, cons
 // ---------------------------------------------------------------------------
 template <int KIND>
 __device__ __forceinline__ void p2_tile(const TensorDev& d, int rb, int cb, const StepConsts& hc,
-                                        Shared& sm)
+                                        Shared& sm, unsigned* done_flag = nullptr, unsigned epoch = 0u)
 {
     constexpr int VEC = Traits<KIND>::VEC;
     constexpr int U = (KIND == kF32x8) ? CAME_P12_U / 2 : CAME_P12_U;   // 32 raw registers either way
@@ -658,7 +745,7 @@ __device__ __forceinline__ void p2_tile(const TensorDev& d, int rb, int cb, cons
         }
     }
     acc = block_sum(acc, sm);
-    finalize_kappa(d, rb * d.n_cb + cb, acc, hc.clip_d, sm);
+    finalize_kappa(d, rb * d.n_cb + cb, acc, hc.clip_d, sm, done_flag, epoch);
 }
 
 // ---------------------------------------------------------------------------
@@ -668,7 +755,7 @@ __device__ __forceinline__ void p2_tile(const TensorDev& d, int rb, int cb, cons
 // ---------------------------------------------------------------------------
 template <int KIND>
 __device__ __forceinline__ void p3_tile(const TensorDev& d, int rb, int cb, const StepConsts& hc,
-                                        Shared& sm)
+                                        Shared& sm, unsigned* done_flag = nullptr, unsigned epoch = 0u)
 {
     constexpr int VEC = Traits<KIND>::VEC;
     constexpr int U = CAME_P34_U;
@@ -741,7 +828,8 @@ __device__ __forceinline__ void p3_tile(const TensorDev& d, int rb, int cb, cons
         store_row_partials<U>(rs, rowpart_seg, rbase, q.TY, q.row1, lane);
     }
     write_col_partials<VEC>(d, q, rb, cacc, sm);
-    finalize_factors(d, rb, cb, hc.beta3, hc.omb3, hc.eps2, hc.b1sq, d.R, d.C, d.scal + 2, sm);
+    finalize_factors(d, rb, cb, hc.beta3, hc.omb3, hc.eps2, hc.b1sq, d.R, d.C, d.scal + 2, sm,
+                     done_flag, epoch);
 }
 
 // ---------------------------------------------------------------------------
@@ -879,7 +967,9 @@ __device__ __forceinline__ float load_grad_scalar(const TensorDev& d, long long 
 
 // v_t = beta2 v + (1-beta2)(g^2 + eps1);  partial sum of u^2 = g^2 / v_t;  kappa when complete
 __device__ __forceinline__ void vec_second_moment_chunk(const TensorDev& d, int chunk,
-                                                        const StepConsts& hc, Shared& sm)
+                                                        const StepConsts& hc, Shared& sm,
+                                                        unsigned* done_flag = nullptr,
+                                                        unsigned epoch = 0u)
 {
     const long long i0 = static_cast<long long>(chunk) * kVecChunk + threadIdx.x;
     float g[kVecPerThread], v[kVecPerThread];
@@ -902,7 +992,7 @@ __device__ __forceinline__ void vec_second_moment_chunk(const TensorDev& d, int 
         }
     }
     acc = block_sum(acc, sm);
-    finalize_kappa(d, chunk, acc, hc.clip_d, sm);
+    finalize_kappa(d, chunk, acc, hc.clip_d, sm, done_flag, epoch);
 }
 
 // uhat, m_t, S_t, theta_t (S and the confidence term skipped for kFlagVecNoConf)
@@ -1034,6 +1124,109 @@ k_p34_adafactor_apply(const TensorDev* __restrict__ T, const Tile* __restrict__ 
     pdl_wait_for_previous_grid();
     if (d.ndim == 1) { vec_apply_chunk(d, t.rb, hc); return; }
     CAME_DISPATCH(p34_adafactor_tile, d, t.rb, t.cb, hc)
+}
+
+// ---------------------------------------------------------------------------
+// Pipelined schedule: the whole step in one persistent grid (see the top of this file).
+// `adafactor` selects Algorithm 1 (phase 2 is then the fused momentum + apply pass and there
+// is no phase 3).  `wait_limit_ns` bounds every wait for a flag.
+// ---------------------------------------------------------------------------
+#ifndef CAME_PIPE_MINB
+#define CAME_PIPE_MINB 2
+#endif
+
+// Out-of-line instances of the tile routines for the persistent grid: each gets a register
+// allocation of its own instead of one allocation for the union of twenty-five inlined bodies
+// (which spilled several KB); the descriptor is then read from the caller's frame.
+template <int KIND> __device__ __noinline__ void p1_call(const TensorDev& d, int rb, int cb, const StepConsts& hc, Shared& sm, unsigned epoch) { p1_tile<KIND>(d, rb, cb, hc, sm, d.done + 0, epoch); }
+template <int KIND> __device__ __noinline__ void p2_call(const TensorDev& d, int rb, int cb, const StepConsts& hc, Shared& sm, unsigned epoch) { p2_tile<KIND>(d, rb, cb, hc, sm, d.done + 1, epoch); }
+template <int KIND> __device__ __noinline__ void p3_call(const TensorDev& d, int rb, int cb, const StepConsts& hc, Shared& sm, unsigned epoch) { p3_tile<KIND>(d, rb, cb, hc, sm, d.done + 2, epoch); }
+template <int KIND> __device__ __noinline__ void p4_call(const TensorDev& d, int rb, int cb, const StepConsts& hc) { p4_tile<KIND>(d, rb, cb, hc); }
+template <int KIND> __device__ __noinline__ void p34_call(const TensorDev& d, int rb, int cb, const StepConsts& hc) { p34_adafactor_tile<KIND>(d, rb, cb, hc); }
+__device__ __noinline__ void vec_a_call(const TensorDev& d, int chunk, const StepConsts& hc, Shared& sm, unsigned epoch) { vec_second_moment_chunk(d, chunk, hc, sm, d.done + 1, epoch); }
+__device__ __noinline__ void vec_b_call(const TensorDev& d, int chunk, const StepConsts& hc) { vec_apply_chunk(d, chunk, hc); }
+
+__global__ void __launch_bounds__(kThreads, CAME_PIPE_MINB)
+k_step_pipelined(const TensorDev* __restrict__ T, const Item* __restrict__ items, int nitems,
+                 PipeSync* __restrict__ sync, StepConsts hc, int adafactor,
+                 unsigned long long wait_limit_ns)
+{
+    __shared__ Shared sm;
+    __shared__ unsigned s_ctl[4];          // [0] ticket  [1] epoch of this step  [2] go on?
+    const int tid = threadIdx.x;
+    if (tid == 0) {
+        const unsigned err = load_acquire(&sync->error);
+        s_ctl[2] = (err == 0u);
+        s_ctl[1] = load_acquire(&sync->epoch) + 1u;
+        // a grid that starts with the error word set hands out no ticket and changes nothing
+        s_ctl[0] = (err == 0u) ? atomicAdd(&sync->ticket, 1u) : 0xffffffffu;
+    }
+    __syncthreads();
+    if (!s_ctl[2]) return;
+    const unsigned epoch = s_ctl[1];
+    unsigned ticket = s_ctl[0];
+    bool failed = false;
+
+    while (ticket < static_cast<unsigned>(nitems)) {
+        // the next ticket is requested now and read at the end of this item, so the round trip
+        // of the atomic overlaps the item's work; tickets of one block still increase
+        unsigned next = 0u;
+        if (tid == 0) next = atomicAdd(&sync->ticket, 1u);
+        const Item it = items[ticket];
+        const TensorDev d = T[it.tensor];
+        // tensor-wide results this item needs: P2 <- r,c ; P3 (vector apply) <- kappa ; P4 <- R,C
+        const int need = (it.phase == 0) ? -1 : it.phase - 1;
+        if (need >= 0) {
+            if (tid == 0)
+                s_ctl[2] = wait_for_flag(d.done + need, epoch, &sync->error, &sync->err_item, ticket,
+                                         wait_limit_ns) ? 1u : 0u;
+            __syncthreads();
+            if (!s_ctl[2]) { failed = true; break; }
+        }
+        if (d.ndim == 1) {
+            if (it.phase == 0) vec_a_call(d, it.rb, hc, sm, epoch);
+            else vec_b_call(d, it.rb, hc);
+        } else {
+            switch (it.phase) {
+                case 0: CAME_DISPATCH(p1_call, d, it.rb, it.cb, hc, sm, epoch) break;
+                case 1: CAME_DISPATCH(p2_call, d, it.rb, it.cb, hc, sm, epoch) break;
+                case 2:
+                    if (adafactor) { CAME_DISPATCH(p34_call, d, it.rb, it.cb, hc) }
+                    else { CAME_DISPATCH(p3_call, d, it.rb, it.cb, hc, sm, epoch) }
+                    break;
+                default: CAME_DISPATCH(p4_call, d, it.rb, it.cb, hc) break;
+            }
+        }
+        __syncthreads();                    // the item is done with the shared scratch
+        if (tid == 0) s_ctl[0] = next;
+        __syncthreads();
+        ticket = s_ctl[0];
+    }
+
+    // leave: the last block out re-arms the control block for the next step
+    __syncthreads();
+    if (tid == 0) {
+        __threadfence();
+        const unsigned e = atomicAdd(&sync->exited, 1u);
+        if (e == gridDim.x - 1u) {
+            sync->ticket = 0u;
+            sync->exited = 0u;
+            if (!failed && load_acquire(&sync->error) == 0u) sync->epoch = epoch;
+            __threadfence();
+        }
+    }
+}
+
+// Runs the bounded wait of the pipelined schedule on a flag that nothing ever sets, so that
+// the time-out path can be exercised on its own: words[3] receives 1 if the wait reported a
+// time-out (and set the error word), 0 if it claimed the flag had arrived.
+__global__ void k_wait_probe(unsigned* words /* [0] flag (stays 0) [1] error [2] err_item [3] status */,
+                             unsigned long long limit_ns)
+{
+    if (threadIdx.x == 0 && blockIdx.x == 0) {
+        const bool ok = wait_for_flag(words + 0, 1u, words + 1, words + 2, 7u, limit_ns);
+        words[3] = ok ? 0u : 1u;
+    }
 }
 
 }  // namespace came
