@@ -1153,6 +1153,9 @@ k_step_pipelined(const TensorDev* __restrict__ T, const Item* __restrict__ items
 {
     __shared__ Shared sm;
     __shared__ unsigned s_ctl[4];          // [0] ticket  [1] epoch of this step  [2] go on?
+#ifdef CAME_PIPE_INLINE
+    __shared__ TensorDev s_d;
+#endif
     const int tid = threadIdx.x;
     if (tid == 0) {
         const unsigned err = load_acquire(&sync->error);
@@ -1173,7 +1176,18 @@ k_step_pipelined(const TensorDev* __restrict__ T, const Item* __restrict__ items
         unsigned next = 0u;
         if (tid == 0) next = atomicAdd(&sync->ticket, 1u);
         const Item it = items[ticket];
+#ifdef CAME_PIPE_INLINE
+        // descriptor in shared memory: the inlined tile bodies read its fields from there
+        {
+            const unsigned* src = reinterpret_cast<const unsigned*>(T + it.tensor);
+            unsigned* dst = reinterpret_cast<unsigned*>(&s_d);
+            if (tid < static_cast<int>(sizeof(TensorDev) / 4)) dst[tid] = src[tid];
+        }
+        __syncthreads();
+        const TensorDev& d = s_d;
+#else
         const TensorDev d = T[it.tensor];
+#endif
         // tensor-wide results this item needs: P2 <- r,c ; P3 (vector apply) <- kappa ; P4 <- R,C
         const int need = (it.phase == 0) ? -1 : it.phase - 1;
         if (need >= 0) {
@@ -1183,6 +1197,22 @@ k_step_pipelined(const TensorDev* __restrict__ T, const Item* __restrict__ items
             __syncthreads();
             if (!s_ctl[2]) { failed = true; break; }
         }
+#ifdef CAME_PIPE_INLINE
+        if (d.ndim == 1) {
+            if (it.phase == 0) vec_second_moment_chunk(d, it.rb, hc, sm, d.done + 1, epoch);
+            else vec_apply_chunk(d, it.rb, hc);
+        } else {
+            switch (it.phase) {
+                case 0: CAME_DISPATCH(p1_tile, d, it.rb, it.cb, hc, sm, d.done + 0, epoch) break;
+                case 1: CAME_DISPATCH(p2_tile, d, it.rb, it.cb, hc, sm, d.done + 1, epoch) break;
+                case 2:
+                    if (adafactor) { CAME_DISPATCH(p34_adafactor_tile, d, it.rb, it.cb, hc) }
+                    else { CAME_DISPATCH(p3_tile, d, it.rb, it.cb, hc, sm, d.done + 2, epoch) }
+                    break;
+                default: CAME_DISPATCH(p4_tile, d, it.rb, it.cb, hc) break;
+            }
+        }
+#else
         if (d.ndim == 1) {
             if (it.phase == 0) vec_a_call(d, it.rb, hc, sm, epoch);
             else vec_b_call(d, it.rb, hc);
@@ -1197,6 +1227,7 @@ k_step_pipelined(const TensorDev* __restrict__ T, const Item* __restrict__ items
                 default: CAME_DISPATCH(p4_call, d, it.rb, it.cb, hc) break;
             }
         }
+#endif
         __syncthreads();                    // the item is done with the shared scratch
         if (tid == 0) s_ctl[0] = next;
         __syncthreads();
