@@ -235,7 +235,9 @@ const char* came_phase_name(const came_ctx* ctx, int32_t phase);
  * the GPU (the same routine came_create uses).  Outputs (HOST): elements per
  * thread per load (1, 4 or 8), threads across columns, rows per tile, number of
  * row blocks and column blocks.  `aligned32` says whether param and m are
- * 32-byte aligned; `tile_elems_target` <= 0 selects the default. */
+ * 32-byte aligned; `tile_elems_target` <= 0 selects the default.  (came_create runs a
+ * matrix with cols == 1 as its 1 x rows view, the same memory with the roles of the row and
+ * column factors exchanged, so that every lane has work: ask for the plan of that view.) */
 came_status came_plan_tensor(int64_t rows, int64_t cols, int32_t ndim, int32_t grad_dtype,
                              int32_t aligned32, int64_t tile_elems_target, int32_t* out_vec,
                              int32_t* out_threads_x, int32_t* out_tile_rows, int32_t* out_n_rb,

@@ -588,7 +588,11 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
         const came_tensor& x = t[i];
         const bool a32 = aligned(x.param, 32) && aligned(x.m, 32) &&
                          (x.grad_dtype == CAME_BF16 || aligned(x.grad, 32));
-        Plan p = plan_tensor(x.rows, x.cols, x.ndim, x.grad_dtype, a32, target);
+        // a contiguous n x 1 matrix is the same memory as 1 x n: planned (and run) in that
+        // view, with the factor roles swapped, every lane has a column to work on
+        const bool flat = x.ndim == 2 && x.cols == 1 && x.rows > 1;
+        Plan p = flat ? plan_tensor(1, x.rows, 2, x.grad_dtype, a32, target)
+                      : plan_tensor(x.rows, x.cols, x.ndim, x.grad_dtype, a32, target);
         if (p.n_grp > came::kColGroup) {      // the two-level column reduction covers 16 x 16 row blocks
             delete ctx;
             return fail(nullptr, CAME_ERR_INTERNAL, "tile plan exceeds the column-reduction fan-in");
@@ -611,12 +615,14 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
             }
             for (int rb = 0; rb < p.n_rb; ++rb)
                 for (int cb = 0; cb < p.n_cb; ++cb) tiles.push_back(Tile{i, rb, cb});
-            offs[i].colpart = take(sizeof(float) * static_cast<size_t>(p.n_rb) * x.cols);
-            offs[i].colpart2 = take(sizeof(float) * static_cast<size_t>(p.n_grp) * x.cols);
-            offs[i].rowpart = take(sizeof(float) * static_cast<size_t>(p.n_seg) * x.rows);
-            offs[i].blocksum = take(sizeof(float) * p.n_rb);
-            offs[i].rowscale = take(sizeof(float) * static_cast<size_t>(x.rows));
-            offs[i].colscale = take(sizeof(float) * static_cast<size_t>(x.cols));
+            const size_t vrows = flat ? 1 : static_cast<size_t>(x.rows);      // the view that runs
+            const size_t vcols = flat ? static_cast<size_t>(x.rows) : static_cast<size_t>(x.cols);
+            offs[i].colpart = take(sizeof(float) * static_cast<size_t>(p.n_rb) * vcols);
+            offs[i].colpart2 = take(sizeof(float) * static_cast<size_t>(p.n_grp) * vcols);
+            offs[i].rowpart = take(sizeof(float) * static_cast<size_t>(p.n_seg) * vrows);
+            offs[i].blocksum = take(sizeof(float) * (static_cast<size_t>(p.n_rb) + (flat ? p.n_cb : 0)));
+            offs[i].rowscale = take(sizeof(float) * vrows);
+            offs[i].colscale = take(sizeof(float) * vcols);
         } else {
             const bool conf = !adafactor && !(x.flags & CAME_T_VEC_NO_CONFIDENCE);
             ctx->state_bytes += 4 * (conf ? 3 : 2) * numel;
@@ -719,6 +725,11 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
         d.tx_log2 = lg; d.tr = p.tr; d.n_rb = p.n_rb; d.n_cb = p.n_cb; d.n_seg = p.n_seg;
         d.n_grp = p.n_grp;
         d.n_parts = p.n_parts; d.ndim = x.ndim; d.flags = x.flags;
+        if (x.ndim == 2 && x.cols == 1 && x.rows > 1) {
+            d.rows = 1; d.cols = x.rows;
+            d.r = x.c; d.c = x.r; d.R = x.C; d.C = x.R;
+            d.flags |= came::kFlagSumCols;
+        }
         if (adafactor && x.ndim == 1) d.flags |= came::kFlagVecNoConf;   // Algorithm 1 has no S
         if (!(flags & CAME_CREATE_KEEP_STATE)) {
             const size_t numel = static_cast<size_t>(x.rows) * x.cols;

@@ -75,6 +75,7 @@ struct TensorDev {
     float*       ws_colpart2;  // [n_grp][cols]  sums of kColGroup consecutive row blocks' partials
     float*       ws_rowpart;   // [n_seg][rows]  per-warp-segment row partial sums
     float*       ws_blocksum;  // [n_rb]         sum of the finished row factor over one row block
+                               // (+ [n_cb] sums of the column factor per strip for kFlagSumCols)
     float*       ws_usq;       // [n_parts]      per-tile partial sums of u^2
     float*       ws_rowscale;  // [rows]  rsqrt of the row factor last finished (r_t, then R_t)
     float*       ws_colscale;  // [cols]  rsqrt of the column factor last finished (c_t, then C_t)
@@ -126,6 +127,10 @@ struct StepConsts {
 
 constexpr unsigned kFlagNoWd = 1u << 0;
 constexpr unsigned kFlagVecNoConf = 1u << 1;
+// Internal: the tensor is an n x 1 matrix handled as its 1 x n view (same memory) with the
+// row and column factors swapped, so that all lanes work; the normaliser 1_n^T r of
+// Algorithm 2 is then the sum of the view's COLUMN factor.
+constexpr unsigned kFlagSumCols = 1u << 8;
 
 // ---------------------------------------------------------------------------
 // loads / stores
@@ -470,6 +475,19 @@ __device__ __forceinline__ void finalize_factors(const TensorDev& d, int rb, int
                 }
             }
             if (tid == 0) d.cnt[d.n_rb + cb] = 0u;
+            if (d.flags & kFlagSumCols) {
+                // this strip's share of the normaliser (the values just stored, by the threads
+                // that stored them; fixed order: thread stride, warp tree, warps 0..7)
+                float cs = 0.f;
+                if (d.vec >= 4) {
+                    for (long long col = col0 + 4 * tid; col < col1; col += 4 * kThreads)
+                        cs += (colfac[col] + colfac[col + 1]) + (colfac[col + 2] + colfac[col + 3]);
+                } else {
+                    for (long long col = col0 + tid; col < col1; col += kThreads) cs += colfac[col];
+                }
+                cs = block_sum(cs, sm);
+                if (tid == 0) d.ws_blocksum[d.n_rb + cb] = cs;
+            }
         }
     }
     const unsigned done = (last_r ? 1u : 0u) + (last_c ? 1u : 0u);
@@ -484,7 +502,9 @@ __device__ __forceinline__ void finalize_factors(const TensorDev& d, int rb, int
     if (sm.flag[2]) {
         __threadfence();
         double s = 0.0;
-        for (int k = tid; k < d.n_rb; k += kThreads) s += static_cast<double>(__ldcg(d.ws_blocksum + k));
+        const int k0 = (d.flags & kFlagSumCols) ? d.n_rb : 0;
+        const int k1 = (d.flags & kFlagSumCols) ? d.n_rb + d.n_cb : d.n_rb;
+        for (int k = k0 + tid; k < k1; k += kThreads) s += static_cast<double>(__ldcg(d.ws_blocksum + k));
         s = block_sum(s, sm);
         if (tid == 0) {
             *sqrt_sum = static_cast<float>(sqrt(s));
