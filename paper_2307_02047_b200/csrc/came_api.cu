@@ -340,7 +340,7 @@ came_status launch_step(came_ctx* ctx, const came_hparams* hp, cudaStream_t stre
         const bool prof = ctx->profiling && !ctx->prof_ev.empty();
         cudaEvent_t* ev = prof ? &ctx->prof_ev[(ctx->prof_count % kProfSlots) * (kMaxPhases + 1)] : nullptr;
         if (ev) cudaEventRecord(ev[0], stream);
-        came::k_step_pipelined<<<ctx->pipe_grid, came::kThreads, 0, stream>>>(
+        came::k_step_pipelined<<<ctx->pipe_grid, came::kPipeThreads, 0, stream>>>(
             ctx->d_table, ctx->d_items, ctx->n_items, ctx->d_sync, hc, ctx->adafactor ? 1 : 0,
             ctx->pipe_wait_ns);
         if (ev) cudaEventRecord(ev[1], stream);
@@ -674,7 +674,7 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
         int sms = 0, per_sm = 0;
         CAME_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device), "cudaDeviceGetAttribute");
         CAME_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, came::k_step_pipelined,
-                                                               came::kThreads, 0), "occupancy query");
+                                                               came::kPipeThreads, 0), "occupancy query");
         ctx->pipe_grid = std::max(1, std::min(ctx->n_items, sms * std::max(per_sm, 1)));
         ctx->pipe_wait_ns = static_cast<unsigned long long>(g_pipe_wait_ns > 0 ? g_pipe_wait_ns
                                                                                 : kPipeWaitNsDefault);

@@ -55,7 +55,8 @@ namespace came {
 #define CAME_P34_U 4
 #endif
 
-constexpr int kThreads = 256;
+constexpr int kThreads = 256;          // threads that work on a tile
+constexpr int kHelperThreads = 32;     // pipelined grid only: one more warp that runs ahead
 constexpr int kVecPerThread = 4;
 constexpr int kVecChunk = kThreads * kVecPerThread;   // vector elements per tile (one block)
 constexpr int kColGroup = 16;         // row blocks per group in the two-level column reduction
@@ -205,6 +206,11 @@ __device__ __forceinline__ void store_bf16(uint16_t* p, const float (&x)[VEC])
 // ---------------------------------------------------------------------------
 // block-level helpers (deterministic: fixed shuffle tree, fixed warp order)
 // ---------------------------------------------------------------------------
+// Barrier over the kThreads threads that work on a tile (hardware barrier 1).  In the phase
+// kernels these are all threads of the block; the pipelined grid has one more warp that must
+// not take part.
+__device__ __forceinline__ void block_sync() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+static_assert(kThreads == 256, "block_sync names the thread count");
 __device__ __forceinline__ float warp_sum(float v)
 {
 #pragma unroll
@@ -225,14 +231,14 @@ struct Shared {
     int    flag[4];
 };
 
-// Sum over the block; result valid in every thread.  Two barriers.
+// Sum over the tile's threads; result valid in every one of them.  Two barriers.
 template <typename T>
 __device__ __forceinline__ T block_sum(T v, Shared& sm)
 {
     v = warp_sum(v);
-    __syncthreads();
+    block_sync();
     if ((threadIdx.x & 31) == 0) sm.red[threadIdx.x >> 5] = static_cast<double>(v);
-    __syncthreads();
+    block_sync();
     double s = 0.0;
 #pragma unroll
     for (int w = 0; w < kThreads / 32; ++w) s += sm.red[w];
@@ -372,14 +378,14 @@ __device__ __forceinline__ void finalize_factors(const TensorDev& d, int rb, int
     const int grp_size = min(kColGroup, d.n_rb - grp * kColGroup);
     unsigned* const cnt_grp = d.cnt + d.n_rb + d.n_cb + 2;
     __threadfence();
-    __syncthreads();
+    block_sync();
     if (tid == 0) {
         const unsigned a = atomicAdd(&d.cnt[rb], 1u);
         const unsigned b = atomicAdd(&cnt_grp[grp * d.n_cb + cb], 1u);
         sm.flag[0] = (a == static_cast<unsigned>(d.n_cb - 1));
         sm.flag[1] = (b == static_cast<unsigned>(grp_size - 1));
     }
-    __syncthreads();
+    block_sync();
     const bool last_r = sm.flag[0] != 0, last_g = sm.flag[1] != 0;
     if (!last_r && !last_g) return;
     __threadfence();
@@ -442,13 +448,13 @@ __device__ __forceinline__ void finalize_factors(const TensorDev& d, int rb, int
             }
         }
         __threadfence();
-        __syncthreads();
+        block_sync();
         if (tid == 0) {
             cnt_grp[grp * d.n_cb + cb] = 0u;
             const unsigned c = atomicAdd(&d.cnt[d.n_rb + cb], 1u);
             sm.flag[1] = (c == static_cast<unsigned>(d.n_grp - 1));
         }
-        __syncthreads();
+        block_sync();
         last_c = sm.flag[1] != 0;
         if (last_c) {
             // level 2: the strip's group partials -> EMA, factor and its rsqrt
@@ -493,12 +499,12 @@ __device__ __forceinline__ void finalize_factors(const TensorDev& d, int rb, int
     const unsigned done = (last_r ? 1u : 0u) + (last_c ? 1u : 0u);
     if (done == 0u) return;
     __threadfence();
-    __syncthreads();
+    block_sync();
     if (tid == 0) {
         const unsigned a = atomicAdd(&d.cnt[d.n_rb + d.n_cb], done);
         sm.flag[2] = (a + done == static_cast<unsigned>(d.n_rb + d.n_cb));
     }
-    __syncthreads();
+    block_sync();
     if (sm.flag[2]) {
         __threadfence();
         double s = 0.0;
@@ -523,12 +529,12 @@ __device__ __forceinline__ void finalize_kappa(const TensorDev& d, int part, flo
     const int tid = threadIdx.x;
     if (tid == 0) d.ws_usq[part] = partial;
     __threadfence();
-    __syncthreads();
+    block_sync();
     if (tid == 0) {
         const unsigned a = atomicAdd(&d.cnt[d.n_rb + d.n_cb + 1], 1u);
         sm.flag[3] = (a == static_cast<unsigned>(d.n_parts - 1));
     }
-    __syncthreads();
+    block_sync();
     if (!sm.flag[3]) return;
     __threadfence();
     double s = 0.0;
@@ -632,7 +638,7 @@ __device__ __forceinline__ void write_col_partials(const TensorDev& d, const Geo
         const int TXV = (1 << d.tx_log2) * VEC;
 #pragma unroll
         for (int v = 0; v < VEC; ++v) sm.colred[q.ty * TXV + q.tx * VEC + v] = cacc[v];
-        __syncthreads();
+        block_sync();
         if (q.ty != 0) return;
 #pragma unroll
         for (int v = 0; v < VEC; ++v) {
@@ -664,12 +670,12 @@ __device__ __forceinline__ void store_row_partials(float (&rs)[U], float* __rest
 // ---------------------------------------------------------------------------
 // P1 (Algorithm 2: r_t, c_t): row and column sums of g^2
 // ---------------------------------------------------------------------------
-template <int KIND>
+template <int KIND, int UU = 0>
 __device__ __forceinline__ void p1_tile(const TensorDev& d, int rb, int cb, const StepConsts& hc,
                                         Shared& sm, unsigned* done_flag = nullptr, unsigned epoch = 0u)
 {
     constexpr int VEC = Traits<KIND>::VEC;
-    constexpr int U = (KIND == kF32x8) ? CAME_P12_U / 2 : CAME_P12_U;   // 32 raw registers either way
+    constexpr int U = UU > 0 ? UU : ((KIND == kF32x8) ? CAME_P12_U / 2 : CAME_P12_U);   // 32 raw registers either way
     const Geo q = make_geo<VEC>(d, rb, cb);
     const int lane = threadIdx.x & 31;
     const long long stride = static_cast<long long>(q.TY) * d.cols * grad_elem_bytes<KIND>();
@@ -718,12 +724,12 @@ __device__ __forceinline__ void p1_tile(const TensorDev& d, int rb, int cb, cons
 // ---------------------------------------------------------------------------
 // P2 (Algorithm 2: v_t, u_t; Eq. 1): sum of u^2 -> kappa
 // ---------------------------------------------------------------------------
-template <int KIND>
+template <int KIND, int UU = 0>
 __device__ __forceinline__ void p2_tile(const TensorDev& d, int rb, int cb, const StepConsts& hc,
                                         Shared& sm, unsigned* done_flag = nullptr, unsigned epoch = 0u)
 {
     constexpr int VEC = Traits<KIND>::VEC;
-    constexpr int U = (KIND == kF32x8) ? CAME_P12_U / 2 : CAME_P12_U;   // 32 raw registers either way
+    constexpr int U = UU > 0 ? UU : ((KIND == kF32x8) ? CAME_P12_U / 2 : CAME_P12_U);   // 32 raw registers either way
     const Geo q = make_geo<VEC>(d, rb, cb);
     const long long stride = static_cast<long long>(q.TY) * d.cols * grad_elem_bytes<KIND>();
     const char* gp = static_cast<const char*>(d.g) +
@@ -773,12 +779,12 @@ __device__ __forceinline__ void p2_tile(const TensorDev& d, int rb, int cb, cons
 // With e = uhat_t - m_{t-1}:  m_t = m_{t-1} + (1-beta1) e  and  uhat_t - m_t = beta1 e,
 // so U_t = beta1^2 e^2; the factor beta1^2 is applied once to the finished sums.
 // ---------------------------------------------------------------------------
-template <int KIND>
+template <int KIND, int UU = 0>
 __device__ __forceinline__ void p3_tile(const TensorDev& d, int rb, int cb, const StepConsts& hc,
                                         Shared& sm, unsigned* done_flag = nullptr, unsigned epoch = 0u)
 {
     constexpr int VEC = Traits<KIND>::VEC;
-    constexpr int U = CAME_P34_U;
+    constexpr int U = UU > 0 ? UU : CAME_P34_U;
     const Geo q = make_geo<VEC>(d, rb, cb);
     const int lane = threadIdx.x & 31;
     const long long first = (q.row0 + q.ty) * d.cols + q.col;
@@ -856,11 +862,11 @@ __device__ __forceinline__ void p3_tile(const TensorDev& d, int rb, int cb, cons
 // P4 (Algorithm 2: S_t and the parameter line, plus decoupled decay):
 //   theta -= lr * (m * rsqrt(R_i) * sqrt(sum R) * rsqrt(C_j) + wd * theta)
 // ---------------------------------------------------------------------------
-template <int KIND>
+template <int KIND, int UU = 0>
 __device__ __forceinline__ void p4_tile(const TensorDev& d, int rb, int cb, const StepConsts& hc)
 {
     constexpr int VEC = Traits<KIND>::VEC;
-    constexpr int U = CAME_P34_U;
+    constexpr int U = UU > 0 ? UU : CAME_P34_U;
     const Geo q = make_geo<VEC>(d, rb, cb);
     if (!q.colok) return;
     const long long first = (q.row0 + q.ty) * d.cols + q.col;
@@ -912,12 +918,12 @@ __device__ __forceinline__ void p4_tile(const TensorDev& d, int rb, int cb, cons
 // no further tensor-wide dependency, so momentum and parameter update are one pass:
 //   m_t = m_{t-1} + (1-beta1)(uhat_t - m_{t-1});  theta -= lr * (m_t + wd * theta)
 // ---------------------------------------------------------------------------
-template <int KIND>
+template <int KIND, int UU = 0>
 __device__ __forceinline__ void p34_adafactor_tile(const TensorDev& d, int rb, int cb,
                                                    const StepConsts& hc)
 {
     constexpr int VEC = Traits<KIND>::VEC;
-    constexpr int U = (KIND == kF32x8) ? CAME_P34_U / 2 : CAME_P34_U;   // 24 registers per thread-row there
+    constexpr int U = UU > 0 ? UU : ((KIND == kF32x8) ? CAME_P34_U / 2 : CAME_P34_U);   // 24 registers per thread-row there
     const Geo q = make_geo<VEC>(d, rb, cb);
     if (!q.colok) return;
     const long long first = (q.row0 + q.ty) * d.cols + q.col;
@@ -1150,112 +1156,141 @@ k_p34_adafactor_apply(const TensorDev* __restrict__ T, const Tile* __restrict__ 
 // Pipelined schedule: the whole step in one persistent grid (see the top of this file).
 // `adafactor` selects Algorithm 1 (phase 2 is then the fused momentum + apply pass and there
 // is no phase 3).  `wait_limit_ns` bounds every wait for a flag.
+//
+// A block is kThreads tile threads plus one helper warp.  The helper runs ahead of the tile
+// threads through a two-slot ring in shared memory: it draws the next ticket, fetches the item
+// and its tensor descriptor into the free slot, waits (bounded) for the flag the item needs,
+// and only then hands the slot over.  The round trips to the L2 that each of these steps
+// costs are thus spent while the tile threads stream the previous tile.  Hand-over uses the
+// hardware barriers 2,3 (slot filled) and 4,5 (slot free); every path of the helper ends in a
+// hand-over (a real item, "no more items", or "give up"), so the tile threads never wait for
+// something that does not come.
 // ---------------------------------------------------------------------------
-#ifndef CAME_PIPE_MINB
-#define CAME_PIPE_MINB 2
+#ifndef CAME_PIPE_MAXREG
+#define CAME_PIPE_MAXREG 112               // two blocks of 288 threads per SM
 #endif
+#ifndef CAME_PIPE_U12
+#define CAME_PIPE_U12 0
+#endif
+#ifndef CAME_PIPE_U3
+#define CAME_PIPE_U3 2
+#endif
+#ifndef CAME_PIPE_U4
+#define CAME_PIPE_U4 1
+#endif
+#ifndef CAME_PIPE_U34A
+#define CAME_PIPE_U34A 1
+#endif
+constexpr int kPipeThreads = kThreads + kHelperThreads;
+constexpr int kPipeSlots = 2;
 
-// Out-of-line instances of the tile routines for the persistent grid: each gets a register
-// allocation of its own instead of one allocation for the union of twenty-five inlined bodies
-// (which spilled several KB); the descriptor is then read from the caller's frame.
-template <int KIND> __device__ __noinline__ void p1_call(const TensorDev& d, int rb, int cb, const StepConsts& hc, Shared& sm, unsigned epoch) { p1_tile<KIND>(d, rb, cb, hc, sm, d.done + 0, epoch); }
-template <int KIND> __device__ __noinline__ void p2_call(const TensorDev& d, int rb, int cb, const StepConsts& hc, Shared& sm, unsigned epoch) { p2_tile<KIND>(d, rb, cb, hc, sm, d.done + 1, epoch); }
-template <int KIND> __device__ __noinline__ void p3_call(const TensorDev& d, int rb, int cb, const StepConsts& hc, Shared& sm, unsigned epoch) { p3_tile<KIND>(d, rb, cb, hc, sm, d.done + 2, epoch); }
-template <int KIND> __device__ __noinline__ void p4_call(const TensorDev& d, int rb, int cb, const StepConsts& hc) { p4_tile<KIND>(d, rb, cb, hc); }
-template <int KIND> __device__ __noinline__ void p34_call(const TensorDev& d, int rb, int cb, const StepConsts& hc) { p34_adafactor_tile<KIND>(d, rb, cb, hc); }
-__device__ __noinline__ void vec_a_call(const TensorDev& d, int chunk, const StepConsts& hc, Shared& sm, unsigned epoch) { vec_second_moment_chunk(d, chunk, hc, sm, d.done + 1, epoch); }
-__device__ __noinline__ void vec_b_call(const TensorDev& d, int chunk, const StepConsts& hc) { vec_apply_chunk(d, chunk, hc); }
+struct PipeSlot {
+    TensorDev d;
+    Item it;             // it.phase < 0: -1 = no more items, -2 = a wait ran out
+};
 
-__global__ void __launch_bounds__(kThreads, CAME_PIPE_MINB)
+__device__ __forceinline__ void bar_sync_id(int id, int count)
+{
+    asm volatile("bar.sync %0, %1;" :: "r"(id), "r"(count) : "memory");
+}
+__device__ __forceinline__ void bar_arrive_id(int id, int count)
+{
+    asm volatile("bar.arrive %0, %1;" :: "r"(id), "r"(count) : "memory");
+}
+
+#define CAME_DISPATCH_U(FN, UU, ...)                                       \
+    switch (d.kind) {                                                      \
+        case kF32x4:  FN<kF32x4, UU>(__VA_ARGS__);  break;                 \
+        case kBF16x8: FN<kBF16x8, UU>(__VA_ARGS__); break;                 \
+        case kF32x8:  FN<kF32x8, UU>(__VA_ARGS__);  break;                 \
+        case kF32x1:  FN<kF32x1, UU>(__VA_ARGS__);  break;                 \
+        default:      FN<kBF16x1, UU>(__VA_ARGS__); break;                 \
+    }
+
+__global__ void __maxnreg__(CAME_PIPE_MAXREG)
 k_step_pipelined(const TensorDev* __restrict__ T, const Item* __restrict__ items, int nitems,
                  PipeSync* __restrict__ sync, StepConsts hc, int adafactor,
                  unsigned long long wait_limit_ns)
 {
     __shared__ Shared sm;
-    __shared__ unsigned s_ctl[4];          // [0] ticket  [1] epoch of this step  [2] go on?
-#ifdef CAME_PIPE_INLINE
-    __shared__ TensorDev s_d;
-#endif
+    __shared__ PipeSlot slot[kPipeSlots];
+    __shared__ unsigned s_ctl[2];          // [0] error word at entry  [1] epoch of this step
     const int tid = threadIdx.x;
     if (tid == 0) {
-        const unsigned err = load_acquire(&sync->error);
-        s_ctl[2] = (err == 0u);
+        s_ctl[0] = load_acquire(&sync->error);
         s_ctl[1] = load_acquire(&sync->epoch) + 1u;
-        // a grid that starts with the error word set hands out no ticket and changes nothing
-        s_ctl[0] = (err == 0u) ? atomicAdd(&sync->ticket, 1u) : 0xffffffffu;
     }
-    __syncthreads();
-    if (!s_ctl[2]) return;
+    __syncthreads();                        // all kPipeThreads threads: the only use of barrier 0
+    // a grid that starts with the error word set hands out no ticket and changes nothing
+    if (s_ctl[0] != 0u) return;
     const unsigned epoch = s_ctl[1];
-    unsigned ticket = s_ctl[0];
-    bool failed = false;
 
-    while (ticket < static_cast<unsigned>(nitems)) {
-        // the next ticket is requested now and read at the end of this item, so the round trip
-        // of the atomic overlaps the item's work; tickets of one block still increase
-        unsigned next = 0u;
-        if (tid == 0) next = atomicAdd(&sync->ticket, 1u);
-        const Item it = items[ticket];
-#ifdef CAME_PIPE_INLINE
-        // descriptor in shared memory: the inlined tile bodies read its fields from there
-        {
-            const unsigned* src = reinterpret_cast<const unsigned*>(T + it.tensor);
-            unsigned* dst = reinterpret_cast<unsigned*>(&s_d);
-            if (tid < static_cast<int>(sizeof(TensorDev) / 4)) dst[tid] = src[tid];
+    if (tid >= kThreads) {
+        // ---------------- helper warp ----------------
+        const int lane = tid - kThreads;
+        for (unsigned k = 0;; ++k) {
+            const int s = static_cast<int>(k % kPipeSlots);
+            if (k >= kPipeSlots) bar_sync_id(4 + s, kPipeThreads);      // the tile threads are done with it
+            unsigned ticket = 0u;
+            if (lane == 0) ticket = atomicAdd(&sync->ticket, 1u);
+            ticket = __shfl_sync(0xffffffffu, ticket, 0);
+            int verdict = 0;                                            // 0 go, -1 no more items, -2 give up
+            if (ticket >= static_cast<unsigned>(nitems)) {
+                verdict = -1;
+            } else {
+                const Item it = items[ticket];
+                const unsigned* src = reinterpret_cast<const unsigned*>(T + it.tensor);
+                unsigned* dst = reinterpret_cast<unsigned*>(&slot[s].d);
+                constexpr int kWords = static_cast<int>(sizeof(TensorDev) / 4);
+                for (int w = lane; w < kWords; w += 32) dst[w] = __ldg(src + w);
+                if (lane == 0) slot[s].it = it;
+                __syncwarp();
+                // tensor-wide results the item needs: P2 <- r,c ; P3 (vector apply) <- kappa ; P4 <- R,C
+                if (it.phase > 0) {
+                    int ok = 1;
+                    if (lane == 0)
+                        ok = wait_for_flag(slot[s].d.done + (it.phase - 1), epoch, &sync->error,
+                                           &sync->err_item, ticket, wait_limit_ns) ? 1 : 0;
+                    ok = __shfl_sync(0xffffffffu, ok, 0);
+                    if (!ok) verdict = -2;
+                }
+            }
+            if (verdict != 0 && lane == 0) slot[s].it.phase = verdict;
+            __threadfence_block();
+            bar_arrive_id(2 + s, kPipeThreads);                         // slot filled
+            if (verdict != 0) break;
         }
-        __syncthreads();
-        const TensorDev& d = s_d;
-#else
-        const TensorDev d = T[it.tensor];
-#endif
-        // tensor-wide results this item needs: P2 <- r,c ; P3 (vector apply) <- kappa ; P4 <- R,C
-        const int need = (it.phase == 0) ? -1 : it.phase - 1;
-        if (need >= 0) {
-            if (tid == 0)
-                s_ctl[2] = wait_for_flag(d.done + need, epoch, &sync->error, &sync->err_item, ticket,
-                                         wait_limit_ns) ? 1u : 0u;
-            __syncthreads();
-            if (!s_ctl[2]) { failed = true; break; }
-        }
-#ifdef CAME_PIPE_INLINE
+        return;
+    }
+
+    // ---------------- tile threads ----------------
+    bool failed = false;
+    for (unsigned k = 0;; ++k) {
+        const int s = static_cast<int>(k % kPipeSlots);
+        bar_sync_id(2 + s, kPipeThreads);                               // wait for the helper's hand-over
+        const TensorDev& d = slot[s].d;
+        const int phase = slot[s].it.phase, rb = slot[s].it.rb, cb = slot[s].it.cb;
+        if (phase < 0) { failed = (phase == -2); break; }
         if (d.ndim == 1) {
-            if (it.phase == 0) vec_second_moment_chunk(d, it.rb, hc, sm, d.done + 1, epoch);
-            else vec_apply_chunk(d, it.rb, hc);
+            if (phase == 0) vec_second_moment_chunk(d, rb, hc, sm, d.done + 1, epoch);
+            else vec_apply_chunk(d, rb, hc);
         } else {
-            switch (it.phase) {
-                case 0: CAME_DISPATCH(p1_tile, d, it.rb, it.cb, hc, sm, d.done + 0, epoch) break;
-                case 1: CAME_DISPATCH(p2_tile, d, it.rb, it.cb, hc, sm, d.done + 1, epoch) break;
+            switch (phase) {
+                case 0: CAME_DISPATCH_U(p1_tile, CAME_PIPE_U12, d, rb, cb, hc, sm, d.done + 0, epoch) break;
+                case 1: CAME_DISPATCH_U(p2_tile, CAME_PIPE_U12, d, rb, cb, hc, sm, d.done + 1, epoch) break;
                 case 2:
-                    if (adafactor) { CAME_DISPATCH(p34_adafactor_tile, d, it.rb, it.cb, hc) }
-                    else { CAME_DISPATCH(p3_tile, d, it.rb, it.cb, hc, sm, d.done + 2, epoch) }
+                    if (adafactor) { CAME_DISPATCH_U(p34_adafactor_tile, CAME_PIPE_U34A, d, rb, cb, hc) }
+                    else { CAME_DISPATCH_U(p3_tile, CAME_PIPE_U3, d, rb, cb, hc, sm, d.done + 2, epoch) }
                     break;
-                default: CAME_DISPATCH(p4_tile, d, it.rb, it.cb, hc) break;
+                default: CAME_DISPATCH_U(p4_tile, CAME_PIPE_U4, d, rb, cb, hc) break;
             }
         }
-#else
-        if (d.ndim == 1) {
-            if (it.phase == 0) vec_a_call(d, it.rb, hc, sm, epoch);
-            else vec_b_call(d, it.rb, hc);
-        } else {
-            switch (it.phase) {
-                case 0: CAME_DISPATCH(p1_call, d, it.rb, it.cb, hc, sm, epoch) break;
-                case 1: CAME_DISPATCH(p2_call, d, it.rb, it.cb, hc, sm, epoch) break;
-                case 2:
-                    if (adafactor) { CAME_DISPATCH(p34_call, d, it.rb, it.cb, hc) }
-                    else { CAME_DISPATCH(p3_call, d, it.rb, it.cb, hc, sm, epoch) }
-                    break;
-                default: CAME_DISPATCH(p4_call, d, it.rb, it.cb, hc) break;
-            }
-        }
-#endif
-        __syncthreads();                    // the item is done with the shared scratch
-        if (tid == 0) s_ctl[0] = next;
-        __syncthreads();
-        ticket = s_ctl[0];
+        block_sync();                       // every tile thread is done with the slot and the scratch
+        bar_arrive_id(4 + s, kPipeThreads);                             // slot free
     }
 
     // leave: the last block out re-arms the control block for the next step
-    __syncthreads();
+    block_sync();
     if (tid == 0) {
         __threadfence();
         const unsigned e = atomicAdd(&sync->exited, 1u);
