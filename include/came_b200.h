@@ -319,17 +319,18 @@ enum {
     CAME_TUNE_F32_VEC8 = 4,           /* 1 (default): fp32 gradients are read 8 per thread with
                                          256-bit loads when rows are 32-byte aligned; 0: 4 per
                                          thread (128-bit) */
-    CAME_TUNE_SCHEDULE = 5,           /* schedule of contexts created afterwards: 0 = chosen from
-                                         the tensor sizes, 1 = one grid per phase (four launches),
+    CAME_TUNE_SCHEDULE = 5,           /* schedule of contexts created afterwards: 0 = the default
+                                         (one grid per phase), 1 = one grid per phase (four launches),
                                          2 = pipelined: the whole step is ONE persistent grid whose
                                          blocks draw (tensor, tile, phase) items in an order that
                                          sends L2-sized groups of tensors through the phases one
                                          pipeline stage apart, so a group's gradient is read from
                                          HBM once and its momentum is still in the L2 when the last
-                                         phase reads it.  Same arithmetic, same results. */
-    CAME_TUNE_PIPE_TILE_ELEMS = 6,    /* pipelined schedule: elements per tile (0 = default 8192) */
+                                         phase reads it.  Same arithmetic, same results; measured
+                                         slower than the phase grids on B200, hence not the default. */
+    CAME_TUNE_PIPE_TILE_ELEMS = 6,    /* pipelined schedule: elements per tile (0 = default 32768) */
     CAME_TUNE_PIPE_GROUP_BYTES = 7,   /* pipelined schedule: bytes of gradient + momentum per
-                                         tensor group (0 = default 20 MiB) */
+                                         tensor group (0 = default 48 MiB) */
     CAME_TUNE_PIPE_WAIT_NS = 8,       /* pipelined schedule: limit of every wait for a flag, in
                                          nanoseconds (0 = default 2 s) */
     CAME_TUNE_PIPE_ORDER = 9          /* pipelined schedule: 0 = groups one stage apart (default),

@@ -34,12 +34,9 @@ long long g_pipe_tile_elems = 0;       // came_tune(CAME_TUNE_PIPE_TILE_ELEMS); 
 long long g_pipe_group_bytes = 0;      // came_tune(CAME_TUNE_PIPE_GROUP_BYTES); 0 = default
 long long g_pipe_wait_ns = 0;          // came_tune(CAME_TUNE_PIPE_WAIT_NS); 0 = default (2 s)
 long long g_pipe_order = 0;            // came_tune(CAME_TUNE_PIPE_ORDER)
-constexpr long long kPipeTileElemsDefault = 8192;
-constexpr long long kPipeGroupBytesDefault = 20ll << 20;
+constexpr long long kPipeTileElemsDefault = 32768;
+constexpr long long kPipeGroupBytesDefault = 48ll << 20;
 constexpr long long kPipeWaitNsDefault = 2000000000ll;
-constexpr bool kPipeAutoEnabled = false;              // auto never picks the pipelined grid yet
-constexpr long long kPipeAutoTensorBytes = 40ll << 20;
-constexpr long long kPipeAutoMinTenths = 5;
 
 bool g_f32_vec8 = true;                // came_tune(CAME_TUNE_F32_VEC8)
 inline bool g_f32_vec8_ok(bool bf) { return bf || g_f32_vec8; }
@@ -382,22 +379,14 @@ std::vector<Group> make_groups(const came_ctx* ctx, long long limit, F bytes_of)
     return out;
 }
 
-// Which schedule a new context gets.  came_tune(CAME_TUNE_SCHEDULE) forces one; otherwise the
-// pipelined grid is taken when most of the matrix elements sit in tensors whose gradient and
-// momentum together are small enough for several of them to share the L2.
-bool choose_pipelined(const came_tensor* t, int n)
+// Which schedule a new context gets: one grid per phase unless the pipelined grid is asked
+// for.  (Measured on B200 the pipelined grid is the slower of the two on every workload
+// tried: at 6.5 TB/s the 126 MB L2 turns over in under 20 us, less than the four dependent
+// phases of a tensor group need to pass through it, so the groups either stall on their
+// flags or fall out of the L2.)
+bool choose_pipelined(const came_tensor*, int)
 {
-    if (g_schedule == 1) return false;
-    if (g_schedule == 2) return true;
-    long long small = 0, all = 0;
-    for (int i = 0; i < n; ++i) {
-        if (t[i].ndim != 2) continue;
-        const long long numel = t[i].rows * t[i].cols;
-        const long long resident = numel * (4 + (t[i].grad_dtype == CAME_BF16 ? 2 : 4));
-        all += numel;
-        if (resident <= kPipeAutoTensorBytes) small += numel;
-    }
-    return kPipeAutoEnabled && all > 0 && small * 10 >= all * kPipeAutoMinTenths;
+    return g_schedule == 2;
 }
 
 // Ticket order of the pipelined schedule.  Consecutive tensors form a group until the group's

@@ -1167,13 +1167,13 @@ k_p34_adafactor_apply(const TensorDev* __restrict__ T, const Tile* __restrict__ 
 // something that does not come.
 // ---------------------------------------------------------------------------
 #ifndef CAME_PIPE_MAXREG
-#define CAME_PIPE_MAXREG 112               // two blocks of 288 threads per SM
+#define CAME_PIPE_MAXREG 80                // two blocks of 288 threads per SM (registers are granted per 4 warps)
 #endif
 #ifndef CAME_PIPE_U12
 #define CAME_PIPE_U12 0
 #endif
 #ifndef CAME_PIPE_U3
-#define CAME_PIPE_U3 2
+#define CAME_PIPE_U3 1
 #endif
 #ifndef CAME_PIPE_U4
 #define CAME_PIPE_U4 1
@@ -1189,13 +1189,25 @@ struct PipeSlot {
     Item it;             // it.phase < 0: -1 = no more items, -2 = a wait ran out
 };
 
-__device__ __forceinline__ void bar_sync_id(int id, int count)
+// Hand-over barriers of the ring (all kPipeThreads threads take part: one side arrives, the
+// other waits).  The barrier numbers are literals so that the kernel is charged for the six
+// hardware barriers it uses and no more.
+static_assert(kPipeThreads == 288 && kPipeSlots == 2, "the barrier instructions below name these");
+__device__ __forceinline__ void slot_filled_arrive(int s)
 {
-    asm volatile("bar.sync %0, %1;" :: "r"(id), "r"(count) : "memory");
+    if (s == 0) asm volatile("bar.arrive 2, 288;" ::: "memory"); else asm volatile("bar.arrive 3, 288;" ::: "memory");
 }
-__device__ __forceinline__ void bar_arrive_id(int id, int count)
+__device__ __forceinline__ void slot_filled_wait(int s)
 {
-    asm volatile("bar.arrive %0, %1;" :: "r"(id), "r"(count) : "memory");
+    if (s == 0) asm volatile("bar.sync 2, 288;" ::: "memory"); else asm volatile("bar.sync 3, 288;" ::: "memory");
+}
+__device__ __forceinline__ void slot_free_arrive(int s)
+{
+    if (s == 0) asm volatile("bar.arrive 4, 288;" ::: "memory"); else asm volatile("bar.arrive 5, 288;" ::: "memory");
+}
+__device__ __forceinline__ void slot_free_wait(int s)
+{
+    if (s == 0) asm volatile("bar.sync 4, 288;" ::: "memory"); else asm volatile("bar.sync 5, 288;" ::: "memory");
 }
 
 #define CAME_DISPATCH_U(FN, UU, ...)                                       \
@@ -1228,12 +1240,15 @@ k_step_pipelined(const TensorDev* __restrict__ T, const Item* __restrict__ items
     if (tid >= kThreads) {
         // ---------------- helper warp ----------------
         const int lane = tid - kThreads;
+        unsigned next_ticket = 0u;
+        if (lane == 0) next_ticket = atomicAdd(&sync->ticket, 1u);
         for (unsigned k = 0;; ++k) {
             const int s = static_cast<int>(k % kPipeSlots);
-            if (k >= kPipeSlots) bar_sync_id(4 + s, kPipeThreads);      // the tile threads are done with it
-            unsigned ticket = 0u;
-            if (lane == 0) ticket = atomicAdd(&sync->ticket, 1u);
-            ticket = __shfl_sync(0xffffffffu, ticket, 0);
+            // this item's ticket was requested one round ago; the request for the next one is
+            // issued now, so its round trip overlaps this round's fetches and waits
+            const unsigned ticket = __shfl_sync(0xffffffffu, next_ticket, 0);
+            if (lane == 0 && ticket < static_cast<unsigned>(nitems)) next_ticket = atomicAdd(&sync->ticket, 1u);
+            if (k >= kPipeSlots) slot_free_wait(s);      // the tile threads are done with it
             int verdict = 0;                                            // 0 go, -1 no more items, -2 give up
             if (ticket >= static_cast<unsigned>(nitems)) {
                 verdict = -1;
@@ -1257,7 +1272,7 @@ k_step_pipelined(const TensorDev* __restrict__ T, const Item* __restrict__ items
             }
             if (verdict != 0 && lane == 0) slot[s].it.phase = verdict;
             __threadfence_block();
-            bar_arrive_id(2 + s, kPipeThreads);                         // slot filled
+            slot_filled_arrive(s);
             if (verdict != 0) break;
         }
         return;
@@ -1267,7 +1282,7 @@ k_step_pipelined(const TensorDev* __restrict__ T, const Item* __restrict__ items
     bool failed = false;
     for (unsigned k = 0;; ++k) {
         const int s = static_cast<int>(k % kPipeSlots);
-        bar_sync_id(2 + s, kPipeThreads);                               // wait for the helper's hand-over
+        slot_filled_wait(s);                                            // the helper's hand-over
         const TensorDev& d = slot[s].d;
         const int phase = slot[s].it.phase, rb = slot[s].it.rb, cb = slot[s].it.cb;
         if (phase < 0) { failed = (phase == -2); break; }
@@ -1286,7 +1301,7 @@ k_step_pipelined(const TensorDev* __restrict__ T, const Item* __restrict__ items
             }
         }
         block_sync();                       // every tile thread is done with the slot and the scratch
-        bar_arrive_id(4 + s, kPipeThreads);                             // slot free
+        slot_free_arrive(s);
     }
 
     // leave: the last block out re-arms the control block for the next step
