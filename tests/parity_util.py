@@ -113,20 +113,31 @@ def compare_state(opt, orc, indices=None, p0=None, steps: int = 1) -> dict:
 
 def run_paired(torch, binding, oracle, w: synth.Workload, seed: int, steps: int, check_at,
                flags=None, hparams=None, device="cuda:0", oracle_idx=None, workers: int = 0,
-               algorithm: str = "came", bf16_copy: bool = False):
+               algorithm: str = "came", bf16_copy: bool = False, device_fill_others: bool = False):
     """Step the CUDA path and the oracle side by side; returns {step: worst-error dict}.
 
     ``oracle_idx``: run the oracle on these tensors only (tensors are independent, so each is
     an exact element-by-element check of the full-size GPU run); None = all tensors.
+    ``device_fill_others``: the gradients of the tensors the oracle does NOT follow are drawn on
+    the device (same distribution, other bits) instead of on the host; the followed tensors
+    always get the host-generated bits the oracle sees.  The next step's host gradients are
+    drawn on a background thread while the current step is stepped and compared.
     """
+    from concurrent.futures import ThreadPoolExecutor
     hp = dict(w.hparams if hparams is None else hparams)
     params = synth.make_params(w, seed)
+    sel = list(range(len(params))) if oracle_idx is None else list(oracle_idx)
+    host_idx = sel if (device_fill_others and oracle_idx is not None) else list(range(len(params)))
     dev_p = [torch.from_numpy(p).to(device) for p in params]
-    g0 = synth.make_grads(w, seed, 1, workers=workers)
-    dev_g = [to_torch_grad(torch, g, device) for g in g0]
+    gdt = torch.bfloat16 if w.grad_dtype == synth.BF16 else torch.float32
+    pool = ThreadPoolExecutor(max_workers=1)
+    draw = lambda step: synth.make_grads(w, seed, step, indices=host_idx, workers=workers)
+    pending = pool.submit(draw, 1)
+    dev_g = [torch.empty(t.shape, dtype=gdt, device=device) for t in w.tensors]
+    gen = torch.Generator(device=device)
+    gen.manual_seed(seed)
     opt = binding.CameOptimizer(dev_p, dev_g, flags=flags, bf16_copy=bf16_copy,
                                 create_flags=binding.CAME_CREATE_ADAFACTOR if algorithm == "adafactor" else 0)
-    sel = list(range(len(params))) if oracle_idx is None else list(oracle_idx)
     no_wd = [bool(flags[i] & binding.CAME_T_NO_WEIGHT_DECAY) for i in sel] if flags else ()
     no_conf = [bool(flags[i] & binding.CAME_T_VEC_NO_CONFIDENCE) for i in sel] if flags else ()
     orc = oracle.OracleOptimizer([params[i] for i in sel], no_weight_decay=no_wd,
@@ -134,15 +145,21 @@ def run_paired(torch, binding, oracle, w: synth.Workload, seed: int, steps: int,
     p0 = [params[i] for i in sel]
     del params
     out = {}
+    pos = {i: k for k, i in enumerate(host_idx)}
+    hosted = set(host_idx)
     for step in range(1, steps + 1):
-        grads = g0 if step == 1 else synth.make_grads(w, seed, step, workers=workers)
-        if step > 1:
-            for dg, g in zip(dev_g, grads):
-                dg.copy_(to_torch_grad(torch, g, device))
+        grads = pending.result()
+        pending = pool.submit(draw, step + 1) if step < steps else None
+        for i, dg in enumerate(dev_g):
+            if i in hosted:
+                dg.copy_(to_torch_grad(torch, grads[pos[i]], device))
+            else:
+                dg.normal_(0.0, 1e-3, generator=gen)
         opt.step(**hp)
         gs = float(hp.get("grad_scale", 1.0))       # the step's gradient is gs * buffer
-        orc.step([synth.widen(grads[i]) * gs for i in sel], **hp)
-        g0 = None
+        for j, i in enumerate(sel):                  # one tensor at a time keeps the float64 copies small
+            orc.step_tensor(j, synth.widen(grads[pos[i]]) * gs, **hp)
+        del grads
         if step in check_at:
             torch.cuda.synchronize()
             out[step] = compare_state(opt, orc, None if oracle_idx is None else sel, p0=p0, steps=step)
@@ -151,5 +168,6 @@ def run_paired(torch, binding, oracle, w: synth.Workload, seed: int, steps: int,
                     want = synth.f32_to_bf16_bits(p32.cpu().numpy())
                     got = p16.view(torch.int16).cpu().numpy().view(np.uint16)
                     assert np.array_equal(got, want), "bf16 parameter copy is not RNE of the fp32 result"
+    pool.shutdown()
     opt.close()
     return out

@@ -71,6 +71,31 @@ def test_partition_by_bytes_balances_and_is_deterministic():
     assert sorted(set(partition_by_bytes([7] * 8, 8))) == list(range(8))
 
 
+def test_segment_layout_covers_every_element_once():
+    sys.path.insert(0, ROOT)
+    from paper_2307_02047_b200.sharded import (ALIGN_ELEMS, bucket_pieces, partition_by_bytes,
+                                               segment_layout)
+    numels = [960, 128, 33, 320, 7, 4096, 1]
+    for world in (1, 2, 3):
+        for bucket in (8, 64, 1000, 1 << 20):
+            owner = partition_by_bytes([4 * n for n in numels], world)
+            offset, seg_len, chunk, nb = segment_layout(numels, owner, world, bucket)
+            assert seg_len == nb * chunk and chunk % ALIGN_ELEMS == 0
+            assert all(o % ALIGN_ELEMS == 0 for o in offset)          # 32-byte aligned fp32 views
+            pieces = bucket_pieces(numels, owner, offset, chunk, nb)
+            seen = [0] * len(numels)
+            cells = set()
+            for b, plist in enumerate(pieces):
+                for (i, lo, hi, r, dst) in plist:
+                    assert r == owner[i] and 0 <= lo < hi <= numels[i] and dst + hi - lo <= chunk
+                    assert b * chunk + dst == offset[i] + lo                   # where it sits in the segment
+                    seen[i] += hi - lo
+                    for c in range(dst, dst + hi - lo):
+                        assert (b, r, c) not in cells                          # no two pieces overlap
+                        cells.add((b, r, c))
+            assert seen == numels
+
+
 def _sharded_worker(rank, world, port, q):
     sys.path.insert(0, ROOT)
     import numpy as np
@@ -95,7 +120,9 @@ def _sharded_worker(rank, world, port, q):
             for dst, src in zip(self.p, self.o.p):
                 dst.copy_(torch.from_numpy(src))
 
-    sh = ShardedCame(params, grads, make_local=OracleLocal)
+    # small buckets: several collectives per step, tensors straddling bucket boundaries
+    sh = ShardedCame(params, grads, make_local=OracleLocal, bucket_elems=256)
+    assert sh.n_buckets >= 3 and sh.collectives_per_step == 2 * sh.n_buckets
     for step in (1, 2, 3):
         for i, g in enumerate(grads):       # each rank has its own micro-batch gradient
             g.copy_(torch.from_numpy(synth.widen(synth.make_grad(w, 100 + rank, i, step))))

@@ -65,7 +65,7 @@ def test_llama7b_full_set_sampled_tensors(env):
     idx = [names[n] for n in ("tok_emb", "l0.wq", "l0.w_gate", "l0.w_down", "l0.norm1",
                               "l17.wo", "l31.w_up", "l31.norm2", "norm_f")]
     _gate(run_paired(torch, binding, oracle, w, seed=6, steps=w.steps, check_at=(1, w.steps),
-                     oracle_idx=idx, workers=WORKERS), "llama7b")
+                     oracle_idx=idx, workers=WORKERS, device_fill_others=True), "llama7b")
 
 
 @pytest.mark.parametrize("shape", synth.SWEEP_SHAPES)
