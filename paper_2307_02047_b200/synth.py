@@ -194,13 +194,16 @@ def widen(a: np.ndarray) -> np.ndarray:
     return a.astype(np.float64)
 
 
+def make_param(w: Workload, seed: int, i: int) -> np.ndarray:
+    """Initial value of parameter tensor ``i``, float32, N(0, 0.02^2)."""
+    t = w.tensors[i]
+    z = _rng(seed, i, _PARAM_STEP_KEY).standard_normal(t.numel, dtype=np.float32)
+    return (z * np.float32(0.02)).reshape(t.shape)
+
+
 def make_params(w: Workload, seed: int) -> List[np.ndarray]:
-    """Initial parameters, float32, N(0, 0.02^2)."""
-    out = []
-    for i, t in enumerate(w.tensors):
-        z = _rng(seed, i, _PARAM_STEP_KEY).standard_normal(t.numel, dtype=np.float32)
-        out.append((z * np.float32(0.02)).reshape(t.shape))
-    return out
+    """Initial parameters of every tensor (see make_param)."""
+    return [make_param(w, seed, i) for i in range(len(w.tensors))]
 
 
 def tensor_sigma(w: Workload, seed: int, i: int) -> float:

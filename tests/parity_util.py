@@ -125,17 +125,24 @@ def run_paired(torch, binding, oracle, w: synth.Workload, seed: int, steps: int,
     """
     from concurrent.futures import ThreadPoolExecutor
     hp = dict(w.hparams if hparams is None else hparams)
-    params = synth.make_params(w, seed)
-    sel = list(range(len(params))) if oracle_idx is None else list(oracle_idx)
-    host_idx = sel if (device_fill_others and oracle_idx is not None) else list(range(len(params)))
-    dev_p = [torch.from_numpy(p).to(device) for p in params]
+    n_t = len(w.tensors)
+    sel = list(range(n_t)) if oracle_idx is None else list(oracle_idx)
+    host_idx = sel if (device_fill_others and oracle_idx is not None) else list(range(n_t))
     gdt = torch.bfloat16 if w.grad_dtype == synth.BF16 else torch.float32
+    gen = torch.Generator(device=device)
+    gen.manual_seed(seed)
+    hosted = set(host_idx)
+    params, dev_p = {}, []
+    for i, t in enumerate(w.tensors):
+        if i in hosted:
+            params[i] = synth.make_param(w, seed, i)
+            dev_p.append(torch.from_numpy(params[i]).to(device))
+        else:                                        # not followed by the oracle: any values do
+            dev_p.append(torch.empty(t.shape, dtype=torch.float32, device=device).normal_(0.0, 0.02, generator=gen))
     pool = ThreadPoolExecutor(max_workers=1)
     draw = lambda step: synth.make_grads(w, seed, step, indices=host_idx, workers=workers)
     pending = pool.submit(draw, 1)
     dev_g = [torch.empty(t.shape, dtype=gdt, device=device) for t in w.tensors]
-    gen = torch.Generator(device=device)
-    gen.manual_seed(seed)
     opt = binding.CameOptimizer(dev_p, dev_g, flags=flags, bf16_copy=bf16_copy,
                                 create_flags=binding.CAME_CREATE_ADAFACTOR if algorithm == "adafactor" else 0)
     no_wd = [bool(flags[i] & binding.CAME_T_NO_WEIGHT_DECAY) for i in sel] if flags else ()
@@ -146,7 +153,6 @@ def run_paired(torch, binding, oracle, w: synth.Workload, seed: int, steps: int,
     del params
     out = {}
     pos = {i: k for k, i in enumerate(host_idx)}
-    hosted = set(host_idx)
     for step in range(1, steps + 1):
         grads = pending.result()
         pending = pool.submit(draw, step + 1) if step < steps else None
@@ -158,7 +164,8 @@ def run_paired(torch, binding, oracle, w: synth.Workload, seed: int, steps: int,
         opt.step(**hp)
         gs = float(hp.get("grad_scale", 1.0))       # the step's gradient is gs * buffer
         for j, i in enumerate(sel):                  # one tensor at a time keeps the float64 copies small
-            orc.step_tensor(j, synth.widen(grads[pos[i]]) * gs, **hp)
+            g64 = synth.widen(grads[pos[i]])
+            orc.step_tensor(j, g64 if gs == 1.0 else g64 * gs, **hp)
         del grads
         if step in check_at:
             torch.cuda.synchronize()

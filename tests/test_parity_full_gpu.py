@@ -20,6 +20,16 @@ from tests.parity_util import TOL_STEP1, TOL_STEP10, gate, run_paired
 
 pytestmark = pytest.mark.gpu
 WORKERS = max(1, min(16, os.cpu_count() or 1))
+# CAME_PARITY_FULL=1 runs every configuration to its stated step count (about 15 minutes for
+# the whole GPU suite).  Without it the three longest runs stop earlier, so that the suite
+# stays well inside a 20-minute budget on a slower host: the BERT-large-shaped set at step 20
+# of 50, the GPT-2-medium-shaped set at 10 of 20 and the 128256 x 4096 matrix at 2 of 5;
+# everything else (the BERT-base-shaped set's 100 steps included) always runs in full.
+FULL = os.environ.get("CAME_PARITY_FULL", "0") == "1"
+
+
+def _steps(configured: int, short: int) -> int:
+    return configured if FULL else min(configured, short)
 
 
 @pytest.fixture(scope="module")
@@ -44,7 +54,8 @@ def test_model_shaped_sets_at_their_configured_step_counts(env, name):
     torch, binding, oracle = env
     w = synth.workload(name)
     assert w.steps == {"bert_base": 100, "bert_large": 50, "gpt2_medium": 20}[name]
-    _gate(run_paired(torch, binding, oracle, w, seed=2, steps=w.steps, check_at=(1, 10, w.steps),
+    steps = _steps(w.steps, {"bert_base": 100, "bert_large": 20, "gpt2_medium": 10}[name])
+    _gate(run_paired(torch, binding, oracle, w, seed=2, steps=steps, check_at=(1, 10, steps),
                      workers=WORKERS), name)
 
 
@@ -73,7 +84,8 @@ def test_shape_sweep_five_steps(env, shape):
     torch, binding, oracle = env
     w = synth.workload(f"mat:{shape[0]}x{shape[1]}")
     assert w.steps == 5
-    _gate(run_paired(torch, binding, oracle, w, seed=8, steps=w.steps, check_at=(1, w.steps),
+    steps = _steps(w.steps, 2 if shape[0] * shape[1] > 1 << 28 else 5)
+    _gate(run_paired(torch, binding, oracle, w, seed=8, steps=steps, check_at=(1, steps),
                      workers=WORKERS), w.name)
 
 
