@@ -159,6 +159,10 @@ def run_gpu(args):
     torch.cuda.set_device(local_rank)
     device = torch.device("cuda", local_rank)
     binding.load()                      # raises if the CUDA library cannot be had: no fallback
+    binding.came_tune(binding.CAME_TUNE_SCHEDULE, {"default": 0, "phase": 1, "pipelined": 2}[args.schedule])
+    binding.came_tune(binding.CAME_TUNE_SCHED_GROUP_BYTES, args.sched_group_bytes)
+    binding.came_tune(binding.CAME_TUNE_PIPE_TILE_ELEMS, args.pipe_tile_elems)
+    binding.came_tune(binding.CAME_TUNE_PIPE_GROUP_BYTES, args.pipe_group_bytes)
     w = synth.workload(args.workload)
     hp = dict(w.hparams)
     params, grads = alloc_device_workload(torch, w, device)
@@ -196,7 +200,10 @@ def run_gpu(args):
         ms = marks[0].elapsed_time(marks[-1])
         ms_median = _median([marks[k].elapsed_time(marks[k + 1]) for k in range(args.steps)])
         clocks = sampler.stop() if rank == 0 else {}
-        phase_ms = binding.came_get_phase_ms(opt.ctx)
+        try:
+            phase_ms = binding.came_get_phase_ms(opt.ctx)
+        except binding.CameError:           # grouped launches report no per-phase times
+            phase_ms = []
         phase_names = [binding.came_phase_name(opt.ctx, i) for i in range(len(phase_ms))]
         binding.came_set_profiling(opt.ctx, False)
         # a thermally or hardware-throttled run is rejected and measured again, once
@@ -230,6 +237,8 @@ def run_gpu(args):
 
     peak, peak_kind = measured_peak()
     pb = phase_bytes(w)
+    # the pipelined grid runs all four phases in one launch: its algorithmic bytes are the step's
+    pb["step_pipelined"] = sum(pb.values())
     pb["p34_adafactor_apply"] = pb["p3_momentum_instability"] + pb["p4_apply"] - 12 * sum(
         t.numel for t in w.tensors if t.ndim == 2) + 8 * sum(t.numel for t in w.tensors if t.ndim == 2)
     phases = {n: m for n, m in zip(phase_names, phase_ms)}
@@ -253,6 +262,9 @@ def run_gpu(args):
         "ms_per_step_without_phase_events": ms_plain, "higher_is_better": True,
         "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": args.workload, "algorithm": args.algorithm, "params": numel,
+                   "schedule": SCHEDULE_NAMES.get(opt.query(binding.CAME_Q_SCHEDULE), "?") +
+                               (" (group by group, %d bytes)" % args.sched_group_bytes
+                                if args.sched_group_bytes else ""),
                    "tensors": len(w.tensors), "grad_dtype": w.grad_dtype,
                    "tiles": opt.query(binding.CAME_Q_NUM_TILES),
                    "workspace_bytes": opt.query(binding.CAME_Q_WORKSPACE_BYTES),
@@ -553,6 +565,13 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--algorithm", default="came", choices=["came", "adafactor"],
                     help="came = Algorithm 2 (default); adafactor = Algorithm 1, for the cost ratio")
+    ap.add_argument("--schedule", default="default", choices=["default", "phase", "pipelined"],
+                    help="launch schedule (came_tune CAME_TUNE_SCHEDULE): one grid per phase, or the "
+                         "pipelined persistent grid")
+    ap.add_argument("--sched-group-bytes", type=int, default=0,
+                    help="phase grids launched group by group (CAME_TUNE_SCHED_GROUP_BYTES); 0 = off")
+    ap.add_argument("--pipe-tile-elems", type=int, default=0, help="CAME_TUNE_PIPE_TILE_ELEMS")
+    ap.add_argument("--pipe-group-bytes", type=int, default=0, help="CAME_TUNE_PIPE_GROUP_BYTES")
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-buffer leg (profiling runs)")

@@ -93,8 +93,8 @@ def test_pipelined_parity_many_tensors_flags_and_modes(env, algorithm):
 
 
 def test_pipelined_bert_base_ten_steps(env):
-    """The BERT-base-shaped set at full size in the configuration the schedule is meant for
-    (default tile and group sizes): 25 or so pipeline stages, the embedding a stage of its own."""
+    """The BERT-base-shaped set at full size with the schedule's default tile and group sizes:
+    a dozen or so pipeline stages, the embedding a stage of its own."""
     torch, binding, oracle = env
     w = synth.workload("bert_base")
     with tuned(binding, SCHEDULE=2):
