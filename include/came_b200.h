@@ -153,6 +153,8 @@ enum {
     CAME_Q_SCHEDULE = 10,        /* 0 = one grid per phase, 1 = pipelined persistent grid        */
     CAME_Q_PIPE_GROUPS = 11,     /* pipelined schedule: tensor groups (pipeline stages)          */
     CAME_Q_PIPE_GRID = 12,       /* pipelined schedule: blocks of the persistent grid            */
+    CAME_Q_P1_STREAM_GRID = 14,  /* blocks of the persistent streaming form of the first phase
+                                    (0 = the context uses the one-block-per-tile form)          */
     CAME_Q_DEVICE_ERROR = 13     /* pipelined schedule: 0, or the error word a step left on the
                                     device (low 8 bits: 1 = a bounded wait ran out; upper bits:
                                     the work item that gave up).  SYNCHRONISES the device. */
@@ -333,8 +335,17 @@ enum {
                                          tensor group (0 = default 48 MiB) */
     CAME_TUNE_PIPE_WAIT_NS = 8,       /* pipelined schedule: limit of every wait for a flag, in
                                          nanoseconds (0 = default 2 s) */
-    CAME_TUNE_PIPE_ORDER = 9          /* pipelined schedule: 0 = groups one stage apart (default),
+    CAME_TUNE_PIPE_ORDER = 9,         /* pipelined schedule: 0 = groups one stage apart (default),
                                          1 = each group's phases back to back */
+    CAME_TUNE_P1_STREAM = 10,         /* first phase (r_t, c_t) as a persistent grid that stages the
+                                         gradient through per-thread rings of asynchronous copies
+                                         in shared memory, so that loads stay in flight across
+                                         the per-tile epilogue: 0 = chosen from the tile size
+                                         (default), 1 = never, 2 = whenever the rows load in
+                                         16-byte pieces.  Same sums in the same order: results are
+                                         bit-identical either way. */
+    CAME_TUNE_P1_STREAM_RING = 11     /* batches of 8 x 16 bytes per thread in that ring
+                                         (1..4; 0 = default 2, i.e. 64 KB per block) */
 };
 came_status came_tune(int32_t key, int64_t value);
 

@@ -25,6 +25,7 @@ CAME_CREATE_ADAFACTOR = 2
  CAME_Q_WORKSPACE_BYTES, CAME_Q_NUM_TILES, CAME_Q_LAUNCHES_PER_STEP, CAME_Q_LAST_STEP,
  CAME_Q_NUM_PHASES, CAME_Q_MATRIX_NUMEL, CAME_Q_SCHEDULE, CAME_Q_PIPE_GROUPS, CAME_Q_PIPE_GRID,
  CAME_Q_DEVICE_ERROR) = range(14)
+CAME_Q_P1_STREAM_GRID = 14
 CAME_TUNE_TILE_ELEMS = 0
 CAME_TUNE_SCHED_GROUP_BYTES = 1
 CAME_TUNE_HOST_GROUP_BYTES = 2
@@ -35,6 +36,8 @@ CAME_TUNE_PIPE_TILE_ELEMS = 6
 CAME_TUNE_PIPE_GROUP_BYTES = 7
 CAME_TUNE_PIPE_WAIT_NS = 8
 CAME_TUNE_PIPE_ORDER = 9
+CAME_TUNE_P1_STREAM = 10
+CAME_TUNE_P1_STREAM_RING = 11
 CAME_SCHEDULE_AUTO, CAME_SCHEDULE_PHASE_GRIDS, CAME_SCHEDULE_PIPELINED = 0, 1, 2
 
 EXPORTED = ["came_create", "came_step", "came_step_host", "came_destroy", "came_last_error",

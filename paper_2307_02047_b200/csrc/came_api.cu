@@ -38,6 +38,11 @@ constexpr long long kPipeTileElemsDefault = 32768;
 constexpr long long kPipeGroupBytesDefault = 48ll << 20;
 constexpr long long kPipeWaitNsDefault = 2000000000ll;
 
+int g_p1_stream = 0;                   // came_tune(CAME_TUNE_P1_STREAM): 0 auto, 1 off, 2 on
+int g_p1_stream_ring = 0;              // came_tune(CAME_TUNE_P1_STREAM_RING): batches in the ring; 0 = default
+constexpr int kP1StreamRingDefault = 2;
+constexpr long long kP1StreamAutoTileBytes = 256ll << 10;   // auto: stream when a P1 tile is at most this big
+
 bool g_f32_vec8 = true;                // came_tune(CAME_TUNE_F32_VEC8)
 inline bool g_f32_vec8_ok(bool bf) { return bf || g_f32_vec8; }
 
@@ -113,6 +118,7 @@ struct came_ctx {
     std::vector<TensorDev> host_table;
     TensorDev* d_table = nullptr;
     TensorDev* pinned_table[2] = {nullptr, nullptr};
+    came::StreamTile* pinned_stream[2] = {nullptr, nullptr};
     cudaEvent_t pinned_free[2] = {nullptr, nullptr};
     bool pinned_used[2] = {false, false};
     int pinned_next = 0;
@@ -128,6 +134,13 @@ struct came_ctx {
     size_t ws_bytes = 0, table_bytes = 0;
     long long numel = 0, matrix_numel = 0, state_bytes = 0, stream_bytes = 0, comp_bytes = 0;
     long long last_step = 0;
+    came::StreamTile* d_stream = nullptr;      // streaming P1: the matrix tiles its ring can serve
+    std::vector<came::StreamTile> h_stream;
+    std::vector<long long> stream_goff;        // byte offset of every stream tile inside its gradient
+    int n_stream = 0;
+    Tile* d_others = nullptr;                  // streaming P1: all other tiles (scalar kinds, vector chunks)
+    int n_others = 0;
+    int p1_stream_grid = 0, p1_stream_ring = 0;
     bool pipelined = false;                    // one persistent grid per step instead of one grid per phase
     came::Item* d_items = nullptr;             // pipelined schedule: work items in ticket order
     int n_items = 0;
@@ -249,8 +262,11 @@ void free_ctx(came_ctx* ctx)
     cudaFree(ctx->d_ws);
     cudaFree(ctx->d_items);
     cudaFree(ctx->d_sync);
+    cudaFree(ctx->d_stream);
+    cudaFree(ctx->d_others);
     for (int k = 0; k < 2; ++k) {
         if (ctx->pinned_table[k]) cudaFreeHost(ctx->pinned_table[k]);
+        if (ctx->pinned_stream[k]) cudaFreeHost(ctx->pinned_stream[k]);
         if (ctx->pinned_free[k]) cudaEventDestroy(ctx->pinned_free[k]);
     }
     for (cudaEvent_t e : ctx->prof_ev)
@@ -278,6 +294,18 @@ came_status upload_table(came_ctx* ctx, cudaStream_t stream)
     cudaError_t e = cudaMemcpyAsync(ctx->d_table, ctx->pinned_table[k], ctx->table_bytes,
                                     cudaMemcpyHostToDevice, stream);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaMemcpyAsync(table)");
+    if (ctx->n_stream > 0 && ctx->pinned_stream[k]) {
+        // the streaming P1 reads gradient addresses from its own tile records: rebuild them
+        for (int j = 0; j < ctx->n_stream; ++j) {
+            came::StreamTile r = ctx->h_stream[j];
+            r.g = static_cast<const char*>(ctx->host_table[r.tensor].g) + ctx->stream_goff[j];
+            ctx->h_stream[j] = r;
+            ctx->pinned_stream[k][j] = r;
+        }
+        e = cudaMemcpyAsync(ctx->d_stream, ctx->pinned_stream[k], sizeof(came::StreamTile) * ctx->n_stream,
+                            cudaMemcpyHostToDevice, stream);
+        if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaMemcpyAsync(stream tiles)");
+    }
     e = cudaEventRecord(ctx->pinned_free[k], stream);
     if (e != cudaSuccess) return cuda_fail(ctx, e, "cudaEventRecord(table slot)");
     ctx->pinned_used[k] = true;
@@ -302,6 +330,25 @@ void launch_phase(K kernel, int grid, cudaStream_t stream, const TensorDev* tabl
     cudaLaunchKernelEx(&cfg, kernel, table, tiles, ntiles, reverse, hc);
 }
 
+// The streaming form of P1 over the whole tile list (persistent grid, dynamic shared memory
+// for the copy ring), launched like the other phase kernels.
+void launch_p1_stream(const came_ctx* ctx, const StepConsts& hc, cudaStream_t stream)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(static_cast<unsigned>(ctx->p1_stream_grid));
+    cfg.blockDim = dim3(came::kThreads);
+    cfg.dynamicSmemBytes = static_cast<size_t>(ctx->p1_stream_ring) * came::kStreamSlots * came::kThreads * 16;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = g_use_pdl ? 1 : 0;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, came::k_p1_stream, static_cast<const TensorDev*>(ctx->d_table),
+                       static_cast<const came::StreamTile*>(ctx->d_stream), ctx->n_stream,
+                       static_cast<const Tile*>(ctx->d_others), ctx->n_others, ctx->p1_stream_ring, hc);
+}
+
 // Enqueue the kernels of one step for the tensors of `g` (all phases, in dependency order).
 // `ev` (may be NULL) receives one event before the first kernel and one after each kernel.
 int launch_range(const came_ctx* ctx, const StepConsts& hc, cudaStream_t stream, const Group& g,
@@ -313,7 +360,10 @@ int launch_range(const came_ctx* ctx, const StepConsts& hc, cudaStream_t stream,
     const Tile* tiles = ctx->d_tiles + g.tile0;
     mark(0);
     if (nt > 0) {
-        launch_phase(came::k_p1_reduce_g2, nt, stream, ctx->d_table, tiles, nt, 0, hc);
+        if (ctx->p1_stream_grid > 0 && g.tile0 == 0 && g.tile1 == ctx->n_tiles)
+            launch_p1_stream(ctx, hc, stream);
+        else
+            launch_phase(came::k_p1_reduce_g2, nt, stream, ctx->d_table, tiles, nt, 0, hc);
         mark(++iv);
         launch_phase(came::k_p2_sum_u2, nt, stream, ctx->d_table, tiles, nt, 1, hc);
         mark(++iv);
@@ -498,6 +548,8 @@ came_status came_tune(int32_t key, int64_t value)
         case CAME_TUNE_PDL: g_use_pdl = value != 0; break;
         case CAME_TUNE_F32_VEC8: g_f32_vec8 = value != 0; break;
         case CAME_TUNE_HOST_GROUP_BYTES: g_host_group_bytes = value > 0 ? value : (1ll << 30); break;
+        case CAME_TUNE_P1_STREAM: if (value > 2) return CAME_ERR_UNSUPPORTED; g_p1_stream = static_cast<int>(value); break;
+        case CAME_TUNE_P1_STREAM_RING: if (value > came::kStreamMaxBatches) return CAME_ERR_UNSUPPORTED; g_p1_stream_ring = static_cast<int>(value); break;
         case CAME_TUNE_SCHEDULE: if (value > 2) return CAME_ERR_UNSUPPORTED; g_schedule = static_cast<int>(value); break;
         case CAME_TUNE_PIPE_TILE_ELEMS: g_pipe_tile_elems = value; break;
         case CAME_TUNE_PIPE_GROUP_BYTES: g_pipe_group_bytes = value; break;
@@ -731,6 +783,66 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
             }
         }
     }
+    // ---- streaming P1: tile records for the matrices whose rows load in 16-byte pieces ---------
+    if (g_p1_stream != 1) {
+        std::vector<Tile> others;
+        long long stream_bytes = 0;
+        bool fits = true;
+        for (const Tile& tl : tiles) {
+            const TensorDev& d = ctx->host_table[tl.tensor];
+            const bool ring_kind = d.ndim == 2 && (d.kind == came::kF32x4 || d.kind == came::kBF16x8 ||
+                                                   d.kind == came::kF32x8);
+            if (!ring_kind) { others.push_back(tl); continue; }
+            if (d.cols >= (1ll << 31)) { fits = false; break; }
+            const long long sw = (1ll << d.tx_log2) * d.vec;
+            const long long row0 = static_cast<long long>(tl.rb) * d.tr, col0 = static_cast<long long>(tl.cb) * sw;
+            const int esz = d.kind == came::kBF16x8 ? 2 : 4;
+            came::StreamTile r;
+            std::memset(&r, 0, sizeof r);
+            const long long goff = (row0 * d.cols + col0) * esz;
+            r.g = static_cast<const char*>(d.g) + goff;
+            r.rowpart = d.ws_rowpart + static_cast<long long>(tl.cb) * ((1 << d.tx_log2) / 32) * d.rows + row0;
+            r.rows = d.rows;
+            r.tensor = tl.tensor; r.rb = tl.rb; r.cb = tl.cb;
+            r.nrows = static_cast<int>(std::min<long long>(d.rows, row0 + d.tr) - row0);
+            r.ncols = static_cast<int>(std::min<long long>(d.cols - col0, sw));
+            r.cols = static_cast<int>(d.cols);
+            r.kind_tx = d.kind | (d.tx_log2 << 8);
+            ctx->h_stream.push_back(r);
+            ctx->stream_goff.push_back(goff);
+            stream_bytes += static_cast<long long>(r.nrows) * r.ncols * esz;
+        }
+        const long long n_st = static_cast<long long>(ctx->h_stream.size());
+        const bool want = fits && n_st > 0 &&
+                          (g_p1_stream == 2 || stream_bytes / n_st <= kP1StreamAutoTileBytes);
+        if (want) {
+            ctx->n_stream = static_cast<int>(n_st);
+            ctx->n_others = static_cast<int>(others.size());
+            ctx->p1_stream_ring = std::min(came::kStreamMaxBatches,
+                                           std::max(1, g_p1_stream_ring > 0 ? g_p1_stream_ring : kP1StreamRingDefault));
+            const size_t ring_bytes = static_cast<size_t>(ctx->p1_stream_ring) * came::kStreamSlots * came::kThreads * 16;
+            CAME_TRY(cudaFuncSetAttribute(came::k_p1_stream, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          static_cast<int>(ring_bytes)), "cudaFuncSetAttribute(ring)");
+            int sms = 0, per_sm = 0;
+            CAME_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device), "cudaDeviceGetAttribute");
+            CAME_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, came::k_p1_stream, came::kThreads,
+                                                                   ring_bytes), "occupancy query");
+            ctx->p1_stream_grid = std::max(1, std::min(std::max(ctx->n_stream, ctx->n_others), sms * std::max(per_sm, 1)));
+            CAME_TRY(cudaMalloc(&ctx->d_stream, sizeof(came::StreamTile) * ctx->n_stream), "cudaMalloc(stream tiles)");
+            CAME_TRY(cudaMemcpy(ctx->d_stream, ctx->h_stream.data(), sizeof(came::StreamTile) * ctx->n_stream,
+                                cudaMemcpyHostToDevice), "cudaMemcpy(stream tiles)");
+            CAME_TRY(cudaMalloc(&ctx->d_others, sizeof(Tile) * std::max<size_t>(others.size(), 1)), "cudaMalloc(other tiles)");
+            if (!others.empty())
+                CAME_TRY(cudaMemcpy(ctx->d_others, others.data(), sizeof(Tile) * others.size(),
+                                    cudaMemcpyHostToDevice), "cudaMemcpy(other tiles)");
+            for (int k = 0; k < 2; ++k)
+                CAME_TRY(cudaMallocHost(&ctx->pinned_stream[k], sizeof(came::StreamTile) * ctx->n_stream),
+                         "cudaMallocHost(stream tiles)");
+        } else {
+            ctx->h_stream.clear();
+            ctx->stream_goff.clear();
+        }
+    }
     CAME_TRY(cudaMemcpy(ctx->d_table, ctx->host_table.data(), ctx->table_bytes,
                         cudaMemcpyHostToDevice), "cudaMemcpy(table)");
     CAME_TRY(cudaDeviceSynchronize(), "cudaDeviceSynchronize");
@@ -850,6 +962,7 @@ came_status came_query(const came_ctx* ctx, int32_t what, int64_t* out)
         case CAME_Q_WORKSPACE_BYTES:
             *out = static_cast<int64_t>(ctx->ws_bytes + ctx->table_bytes + sizeof(Tile) * ctx->n_tiles +
                                         sizeof(came::Item) * ctx->n_items +
+                                        sizeof(came::StreamTile) * ctx->n_stream + sizeof(Tile) * ctx->n_others +
                                         (ctx->d_sync ? sizeof(came::PipeSync) : 0));
             break;
         case CAME_Q_NUM_TILES: *out = ctx->n_tiles; break;
@@ -860,6 +973,7 @@ came_status came_query(const came_ctx* ctx, int32_t what, int64_t* out)
             *out = ctx->pipelined ? 1 : (ctx->adafactor ? 3 : 4); break;
         case CAME_Q_MATRIX_NUMEL: *out = ctx->matrix_numel; break;
         case CAME_Q_SCHEDULE: *out = ctx->pipelined ? 1 : 0; break;
+        case CAME_Q_P1_STREAM_GRID: *out = ctx->pipelined ? 0 : ctx->p1_stream_grid; break;
         case CAME_Q_PIPE_GROUPS: *out = ctx->pipe_groups; break;
         case CAME_Q_PIPE_GRID: *out = ctx->pipe_grid; break;
         case CAME_Q_DEVICE_ERROR: {
