@@ -71,7 +71,8 @@ typedef enum {
     CAME_ERR_OOM = 8,         /* host or device allocation failed */
     CAME_ERR_CUDA = 9,        /* a CUDA runtime call failed; see came_last_error */
     CAME_ERR_INTERNAL = 10,
-    CAME_ERR_UNSUPPORTED = 11 /* request outside what this entry point handles */
+    CAME_ERR_UNSUPPORTED = 11,/* request outside what this entry point handles */
+    CAME_ERR_OVERLAP = 12     /* two of the buffers passed to came_create share memory */
 } came_status;
 
 typedef enum { CAME_F32 = 0, CAME_BF16 = 1 } came_dtype;   /* gradient storage type */
@@ -93,7 +94,10 @@ enum {
 };
 
 /* One parameter tensor.  All pointers are DEVICE pointers, 16-byte aligned,
- * to contiguous, non-overlapping buffers that stay valid until came_destroy. */
+ * to contiguous, non-overlapping buffers that stay valid until came_destroy
+ * (came_create compares every buffer of every tensor with every other and answers
+ * CAME_ERR_OVERLAP if two share a byte; gradient pointers swapped in later through
+ * came_step are the caller's responsibility). */
 typedef struct {
     float*       param;   /* fp32 [rows*cols], row-major; updated in place              */
     const void*  grad;    /* grad_dtype [rows*cols], same layout; read only             */
@@ -302,7 +306,8 @@ came_status came_factor_update_static_plan(const void* grad, int32_t grad_dtype,
                                            double beta2, double eps1, int32_t device,
                                            int32_t* out_vec, int64_t* out_scratch_bytes);
 
-/* Process-wide tuning knobs, read by later came_create calls.  CAME_TUNE_TILE_ELEMS:
+/* Process-wide tuning knobs, read by later came_create calls (plain globals: set them from
+ * one thread, before the contexts they are meant for are created).  CAME_TUNE_TILE_ELEMS:
  * elements per matrix tile (0 restores the default, which scales with the size
  * of the parameter set).  They change scheduling only, never results beyond the
  * order of the partial sums. */
@@ -340,10 +345,11 @@ enum {
     CAME_TUNE_P1_STREAM = 10,         /* first phase (r_t, c_t) as a persistent grid that stages the
                                          gradient through per-thread rings of asynchronous copies
                                          in shared memory, so that loads stay in flight across
-                                         the per-tile epilogue: 0 = chosen from the tile size
-                                         (default), 1 = never, 2 = whenever the rows load in
-                                         16-byte pieces.  Same sums in the same order: results are
-                                         bit-identical either way. */
+                                         the per-tile epilogue: 0 or 1 = off (default), 2 = for
+                                         every matrix whose rows load in 16-byte pieces.  Same
+                                         sums in the same order: results are bit-identical either
+                                         way.  Measured slower on B200 (the phase is bound by
+                                         instruction issue once the latency is hidden), hence off. */
     CAME_TUNE_P1_STREAM_RING = 11     /* batches of 8 x 16 bytes per thread in that ring
                                          (1..4; 0 = default 2, i.e. 64 KB per block) */
 };

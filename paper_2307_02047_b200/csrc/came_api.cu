@@ -38,10 +38,9 @@ constexpr long long kPipeTileElemsDefault = 32768;
 constexpr long long kPipeGroupBytesDefault = 48ll << 20;
 constexpr long long kPipeWaitNsDefault = 2000000000ll;
 
-int g_p1_stream = 0;                   // came_tune(CAME_TUNE_P1_STREAM): 0 auto, 1 off, 2 on
+int g_p1_stream = 0;                   // came_tune(CAME_TUNE_P1_STREAM): 0 default (off), 1 off, 2 on
 int g_p1_stream_ring = 0;              // came_tune(CAME_TUNE_P1_STREAM_RING): batches in the ring; 0 = default
 constexpr int kP1StreamRingDefault = 2;
-constexpr long long kP1StreamAutoTileBytes = 256ll << 10;   // auto: stream when a P1 tile is at most this big
 
 bool g_f32_vec8 = true;                // came_tune(CAME_TUNE_F32_VEC8)
 inline bool g_f32_vec8_ok(bool bf) { return bf || g_f32_vec8; }
@@ -206,6 +205,47 @@ came_status validate_tensor(const came_tensor& t, int i, bool adafactor, std::st
         if (p && !aligned(p, 16)) return err(CAME_ERR_ALIGN, "pointer not 16-byte aligned");
     if ((t.flags & CAME_T_VEC_NO_CONFIDENCE) && t.ndim != 1)
         return err(CAME_ERR_SHAPE, "CAME_T_VEC_NO_CONFIDENCE applies to vectors only");
+    return CAME_OK;
+}
+
+// Every buffer of every tensor must be its own memory: the phases read one tensor's state
+// while they write another's, and the tiles of one buffer are written by different blocks.
+// Sorts all [address, address + bytes) ranges and compares neighbours.
+came_status check_no_overlap(const came_tensor* t, int n, bool adafactor, std::string& msg)
+{
+    struct Range { uintptr_t lo, hi; int tensor; const char* what; };
+    std::vector<Range> rs;
+    rs.reserve(static_cast<size_t>(n) * 8);
+    for (int i = 0; i < n; ++i) {
+        const came_tensor& x = t[i];
+        const unsigned long long numel = static_cast<unsigned long long>(x.rows) * x.cols;
+        const unsigned long long sg = x.grad_dtype == CAME_BF16 ? 2 : 4;
+        auto add = [&](const void* p, unsigned long long bytes, const char* what) {
+            if (p && bytes) rs.push_back(Range{reinterpret_cast<uintptr_t>(p),
+                                               reinterpret_cast<uintptr_t>(p) + bytes, i, what});
+        };
+        add(x.param, 4 * numel, "param");
+        add(x.grad, sg * numel, "grad");
+        add(x.m, 4 * numel, "m");
+        add(x.r, 4ull * x.rows, "r");
+        if (x.ndim == 2) add(x.c, 4ull * x.cols, "c");
+        const bool conf = !adafactor && !(x.ndim == 1 && (x.flags & CAME_T_VEC_NO_CONFIDENCE));
+        if (conf) {
+            add(x.R, 4ull * x.rows, "R");
+            if (x.ndim == 2) add(x.C, 4ull * x.cols, "C");
+        }
+        add(x.param_bf16, 2 * numel, "param_bf16");
+    }
+    std::sort(rs.begin(), rs.end(), [](const Range& a, const Range& b) { return a.lo < b.lo; });
+    for (size_t k = 1; k < rs.size(); ++k) {
+        if (rs[k].lo < rs[k - 1].hi) {
+            char buf[200];
+            std::snprintf(buf, sizeof buf, "buffers overlap: %s of tensor %d and %s of tensor %d",
+                          rs[k - 1].what, rs[k - 1].tensor, rs[k].what, rs[k].tensor);
+            msg = buf;
+            return CAME_ERR_OVERLAP;
+        }
+    }
     return CAME_OK;
 }
 
@@ -530,6 +570,7 @@ const char* came_status_string(came_status s)
         case CAME_ERR_CUDA: return "CAME_ERR_CUDA";
         case CAME_ERR_INTERNAL: return "CAME_ERR_INTERNAL";
         case CAME_ERR_UNSUPPORTED: return "CAME_ERR_UNSUPPORTED";
+        case CAME_ERR_OVERLAP: return "CAME_ERR_OVERLAP";
     }
     return "CAME_ERR_?";
 }
@@ -586,6 +627,10 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
     std::string msg;
     for (int i = 0; i < n; ++i) {
         const came_status s = validate_tensor(t[i], i, adafactor, msg);
+        if (s != CAME_OK) return fail(nullptr, s, msg);
+    }
+    {
+        const came_status s = check_no_overlap(t, n, adafactor, msg);
         if (s != CAME_OK) return fail(nullptr, s, msg);
     }
     int ndev = 0;
@@ -784,9 +829,12 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
         }
     }
     // ---- streaming P1: tile records for the matrices whose rows load in 16-byte pieces ---------
-    if (g_p1_stream != 1) {
+    // (Off unless asked for: measured on B200 the ring hides the memory latency as intended --
+    // long-scoreboard stalls drop from 7.9 to 1.4 cycles per issued instruction -- but P1 then
+    // turns out to be bound by instruction issue, and the ring's extra copy, shared-memory read
+    // and bookkeeping instructions, 1.5x the per-tile form's count, make it 1.5-2x slower.)
+    if (g_p1_stream == 2) {
         std::vector<Tile> others;
-        long long stream_bytes = 0;
         bool fits = true;
         for (const Tile& tl : tiles) {
             const TensorDev& d = ctx->host_table[tl.tensor];
@@ -810,11 +858,9 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
             r.kind_tx = d.kind | (d.tx_log2 << 8);
             ctx->h_stream.push_back(r);
             ctx->stream_goff.push_back(goff);
-            stream_bytes += static_cast<long long>(r.nrows) * r.ncols * esz;
         }
         const long long n_st = static_cast<long long>(ctx->h_stream.size());
-        const bool want = fits && n_st > 0 &&
-                          (g_p1_stream == 2 || stream_bytes / n_st <= kP1StreamAutoTileBytes);
+        const bool want = fits && n_st > 0;
         if (want) {
             ctx->n_stream = static_cast<int>(n_st);
             ctx->n_others = static_cast<int>(others.size());

@@ -1168,6 +1168,12 @@ k_p34_adafactor_apply(const TensorDev* __restrict__ T, const Tile* __restrict__ 
 // anybody else.  Batches, row order and reduction trees are those of p1_tile, hence the
 // identical results.
 //
+// Measured on B200 (BERT-large-shaped set, ncu): the ring does what it is for -- long-scoreboard
+// stalls per issued instruction fall from 7.9 to 1.4 -- but the phase then proves to be bound by
+// instruction issue (about 40 % of peak in both forms), and this form executes 96 M warp
+// instructions where p1_tile executes 63 M (copy, shared-memory read, ring bookkeeping), so it
+// takes 204 us against 132 us.  It is therefore an option (CAME_TUNE_P1_STREAM), not the default.
+//
 // The grid is persistent: block b takes stream tiles b, b + gridDim.x, ...; afterwards it
 // runs the tiles the ring cannot serve (scalar kinds) and the vector chunks through the
 // ordinary routines.
@@ -1480,9 +1486,9 @@ k_step_pipelined(const TensorDev* __restrict__ T, const Item* __restrict__ items
             const unsigned ticket = __shfl_sync(0xffffffffu, next_ticket, 0);
             if (lane == 0 && ticket < static_cast<unsigned>(nitems)) next_ticket = atomicAdd(&sync->ticket, 1u);
             if (k >= kPipeSlots) slot_free_wait(s);      // the tile threads are done with it
-            int verdict = 0;                                            // 0 go, -1 no more items, -2 give up
+            int outcome = 0;                                            // 0 go, -1 no more items, -2 give up
             if (ticket >= static_cast<unsigned>(nitems)) {
-                verdict = -1;
+                outcome = -1;
             } else {
                 const Item it = items[ticket];
                 const unsigned* src = reinterpret_cast<const unsigned*>(T + it.tensor);
@@ -1498,13 +1504,13 @@ k_step_pipelined(const TensorDev* __restrict__ T, const Item* __restrict__ items
                         ok = wait_for_flag(slot[s].d.done + (it.phase - 1), epoch, &sync->error,
                                            &sync->err_item, ticket, wait_limit_ns) ? 1 : 0;
                     ok = __shfl_sync(0xffffffffu, ok, 0);
-                    if (!ok) verdict = -2;
+                    if (!ok) outcome = -2;
                 }
             }
-            if (verdict != 0 && lane == 0) slot[s].it.phase = verdict;
+            if (outcome != 0 && lane == 0) slot[s].it.phase = outcome;
             __threadfence_block();
             slot_filled_arrive(s);
-            if (verdict != 0) break;
+            if (outcome != 0) break;
         }
         return;
     }

@@ -195,3 +195,35 @@ def test_lr_warmup_is_a_linear_ramp_to_the_peak():
     assert f(6e-4, 0.0, 3, 0) == 6e-4
     vals = [f(3e-4, 0.0, t, 100) for t in range(0, 120)]
     assert all(b >= a for a, b in zip(vals, vals[1:])) and max(vals) == 3e-4
+
+
+def test_create_rejects_overlapping_buffers_without_cuda():
+    """Two buffers that share memory are refused before any CUDA call (status 12)."""
+    def wide(base=0x100000, **over):          # a 64 x 64 matrix, buffers 64 KiB apart (param is 16 KiB)
+        f = dict(param=base, grad=base + 0x10000, m=base + 0x20000, r=base + 0x30000,
+                 c=base + 0x40000, R=base + 0x50000, C=base + 0x60000)
+        f.update(over)
+        return binding.came_tensor(f["param"], f["grad"], f["m"], f["r"], f["c"], f["R"], f["C"],
+                                   64, 64, 2, 0, 0, 0)
+    numel_bytes = 4 * 64 * 64
+    for over in (dict(grad=0x100000 + 64),                          # grad starts inside param
+                 dict(m=0x110000 + numel_bytes - 16),               # m starts on grad's last 16 bytes
+                 dict(r=0x120000 + numel_bytes - 16),               # r overlaps the end of m
+                 dict(C=0x130000)):                                 # C on top of r
+        with pytest.raises(binding.CameError) as e:
+            binding.came_create([wide(**over)])
+        assert e.value.status == 12, (over, e.value.status)
+        assert "overlap" in str(e.value)
+    # two tensors sharing one gradient buffer
+    a = wide()
+    b = wide(base=0x800000, grad=0x110000)
+    with pytest.raises(binding.CameError) as e:
+        binding.came_create([a, b])
+    assert e.value.status == 12 and "tensor 0" in str(e.value) and "tensor 1" in str(e.value)
+    # buffers that touch but do not overlap pass this check: the next one to fail is the device's
+    import torch
+    if not torch.cuda.is_available():
+        with pytest.raises(binding.CameError) as e:
+            binding.came_create([wide(grad=0x100000 + numel_bytes)])
+        assert e.value.status == 7
+    assert binding.came_status_string(12) == "CAME_ERR_OVERLAP"
