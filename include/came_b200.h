@@ -157,11 +157,11 @@ enum {
     CAME_Q_SCHEDULE = 10,        /* 0 = one grid per phase, 1 = pipelined persistent grid        */
     CAME_Q_PIPE_GROUPS = 11,     /* pipelined schedule: tensor groups (pipeline stages)          */
     CAME_Q_PIPE_GRID = 12,       /* pipelined schedule: blocks of the persistent grid            */
-    CAME_Q_P1_STREAM_GRID = 14,  /* blocks of the persistent streaming form of the first phase
-                                    (0 = the context uses the one-block-per-tile form)          */
-    CAME_Q_DEVICE_ERROR = 13     /* pipelined schedule: 0, or the error word a step left on the
+    CAME_Q_DEVICE_ERROR = 13,    /* pipelined schedule: 0, or the error word a step left on the
                                     device (low 8 bits: 1 = a bounded wait ran out; upper bits:
                                     the work item that gave up).  SYNCHRONISES the device. */
+    CAME_Q_P1_STREAM_GRID = 14   /* blocks of the persistent streaming form of the first phase
+                                    (0 = the context uses the one-block-per-tile form)          */
 };
 
 /* Algorithm 2, set-up.  Validates `t[0..n)` (HOST array of descriptors holding

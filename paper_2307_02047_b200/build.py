@@ -6,8 +6,9 @@ import subprocess
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 SRC = os.path.join(_HERE, "csrc", "came_api.cu")
-DEPS = [SRC, os.path.join(_HERE, "csrc", "came_kernels.cuh"),
-        os.path.join(os.path.dirname(_HERE), "include", "came_b200.h")]
+DEPS = [SRC] + [os.path.join(_HERE, "csrc", h) for h in
+                ("came_kernels.cuh", "came_pipelined.cuh", "came_stream.cuh")] + \
+       [os.path.join(os.path.dirname(_HERE), "include", "came_b200.h")]
 LIB = os.path.join(_HERE, "libcame_b200.so")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

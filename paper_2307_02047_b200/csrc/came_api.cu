@@ -3,6 +3,8 @@
 // per-step kernel launches.  All arithmetic of Algorithm 2 is in came_kernels.cuh.
 #include "../../include/came_b200.h"
 #include "came_kernels.cuh"
+#include "came_pipelined.cuh"
+#include "came_stream.cuh"
 
 #include <algorithm>
 #include <cmath>
