@@ -227,6 +227,17 @@ came_status came_clear_device_error(came_ctx* ctx, void* cuda_stream);
 came_status came_selftest_wait_timeout(int32_t device, int64_t limit_ns, int32_t* out_timed_out,
                                        int32_t* out_error_word, float* out_elapsed_ms);
 
+/* Debug build only (the library compiled with -DCAME_DEBUG_BOUNDS; paper_2307_02047_b200/build.py
+ * builds it as libcame_b200_debug.so): every tile's index arithmetic is checked on the device
+ * against the tensor's shape and the launch plan before anything is accessed.  A violation
+ * never traps: the offending accesses are masked out and a record is kept on the device.
+ * came_debug_bounds copies that record to `out6` (HOST, six words: code of the first violation
+ * -- 0 none, 1 row block, 2 column block, 3 row-partial segment, 4 vector access past the end
+ * of a row, 5 row range -- then its rb, cb, the tensor's rows and cols, and the number of
+ * violating threads) and synchronises the device.  In the ordinary build it writes zeros and
+ * returns CAME_ERR_UNSUPPORTED. */
+came_status came_debug_bounds(int32_t device, uint32_t* out6);
+
 /* Per-phase device timing.  When enabled, came_step records CUDA events on the
  * caller's stream between its kernels (no synchronisation); switching it on
  * restarts the average.  came_get_phase_ms synchronises on the last recorded

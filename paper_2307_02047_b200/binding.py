@@ -45,7 +45,7 @@ EXPORTED = ["came_create", "came_step", "came_step_host", "came_destroy", "came_
             "came_phase_name", "came_plan_tensor", "came_tune", "came_factor_update_static",
             "came_factor_update_static_plan", "came_required_grad_alignment",
             "came_device_status", "came_lr_warmup", "came_clear_device_error",
-            "came_selftest_wait_timeout"]
+            "came_selftest_wait_timeout", "came_debug_bounds"]
 
 
 class CameError(RuntimeError):
@@ -78,8 +78,39 @@ def load():
     global _lib
     if _lib is not None:
         return _lib
-    path = _build.build()
-    L = ctypes.CDLL(path)
+    _lib = _bind(ctypes.CDLL(_build.build()))
+    return _lib
+
+
+_lib_debug = None
+
+
+def load_debug():
+    """The bounds-checking build of the same library (``-DCAME_DEBUG_BOUNDS``), built on demand."""
+    global _lib_debug
+    if _lib_debug is None:
+        _lib_debug = _bind(ctypes.CDLL(_build.build(debug=True)))
+    return _lib_debug
+
+
+class using_debug_build:
+    """``with using_debug_build():`` routes every call of this module through the
+    bounds-checking build for the duration of the block."""
+
+    def __enter__(self):
+        global _lib
+        load()
+        self.saved = _lib
+        _lib = load_debug()
+        return self
+
+    def __exit__(self, *exc):
+        global _lib
+        _lib = self.saved
+
+
+def _bind(L):
+    """Declare the prototypes of every entry point on a freshly loaded library."""
     vp, i32, i64, u32 = ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_uint32
     L.came_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(came_tensor), i32, i32, u32]
     L.came_create.restype = i32
@@ -124,7 +155,8 @@ def load():
     L.came_selftest_wait_timeout.argtypes = [i32, i64, ctypes.POINTER(i32), ctypes.POINTER(i32),
                                              ctypes.POINTER(ctypes.c_float)]
     L.came_selftest_wait_timeout.restype = i32
-    _lib = L
+    L.came_debug_bounds.argtypes = [i32, ctypes.POINTER(ctypes.c_uint32)]
+    L.came_debug_bounds.restype = i32
     return L
 
 
@@ -257,6 +289,14 @@ def came_selftest_wait_timeout(device: int = 0, limit_ns: int = 1_000_000) -> di
     _check(load().came_selftest_wait_timeout(device, limit_ns, ctypes.byref(a), ctypes.byref(b),
                                              ctypes.byref(ms)))
     return {"timed_out": int(a.value), "error_word": int(b.value), "elapsed_ms": float(ms.value)}
+
+
+def came_debug_bounds(device: int = 0) -> dict:
+    """The device-side record of the bounds-checking build (raises CAME_ERR_UNSUPPORTED, status
+    11, on the ordinary build)."""
+    out = (ctypes.c_uint32 * 6)()
+    _check(load().came_debug_bounds(device, out))
+    return dict(zip(("code", "rb", "cb", "rows", "cols", "threads"), (int(x) for x in out)))
 
 
 def make_hparams(step: int, **kw) -> came_hparams:

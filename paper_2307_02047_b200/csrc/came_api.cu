@@ -1092,6 +1092,24 @@ came_status came_selftest_wait_timeout(int32_t device, int64_t limit_ns, int32_t
     return CAME_OK;
 }
 
+came_status came_debug_bounds(int32_t device, uint32_t* out6)
+{
+    if (!out6) return fail(nullptr, CAME_ERR_NULL, "output pointer is NULL");
+#ifdef CAME_DEBUG_BOUNDS
+    cudaError_t e = cudaSetDevice(device);
+    if (e != cudaSuccess) { cudaGetLastError(); return fail(nullptr, CAME_ERR_DEVICE, "cudaSetDevice failed"); }
+    unsigned h[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+    e = cudaMemcpyFromSymbol(h, came::g_debug_bounds, sizeof h);        // synchronises
+    if (e != cudaSuccess) return cuda_fail(nullptr, e, "cudaMemcpyFromSymbol(debug record)");
+    for (int k = 0; k < 6; ++k) out6[k] = h[k];
+    return CAME_OK;
+#else
+    (void)device;
+    for (int k = 0; k < 6; ++k) out6[k] = 0u;
+    return fail(nullptr, CAME_ERR_UNSUPPORTED, "this library was built without CAME_DEBUG_BOUNDS");
+#endif
+}
+
 came_status came_set_profiling(came_ctx* ctx, int32_t enabled)
 {
     if (!ctx) return CAME_ERR_NULL;

@@ -555,7 +555,31 @@ struct Geo {
     int tx, ty, TY, seg;
     long long col, row0, row1;
     bool colok;
+    bool skip;        // debug build only: the tile indices themselves are out of range
 };
+
+// Debug build (-DCAME_DEBUG_BOUNDS): every tile's geometry is checked against the tensor and
+// the launch plan before anything is accessed.  A violation is recorded in a device error
+// word (first one wins, all are counted) and the offending accesses are masked out; nothing
+// traps, so the context stays usable and the host reads the record afterwards.
+#ifdef CAME_DEBUG_BOUNDS
+enum : unsigned { kDbgRowBlock = 1u, kDbgColBlock = 2u, kDbgSegment = 3u, kDbgVectorTail = 4u, kDbgRowRange = 5u };
+__device__ unsigned g_debug_bounds[8];   // [0] code of the first violation  [1] rb  [2] cb  [3] rows  [4] cols
+                                         // [5] number of violating threads
+__device__ __forceinline__ void debug_report(unsigned code, const TensorDev& d, int rb, int cb)
+{
+    atomicAdd(&g_debug_bounds[5], 1u);
+    if (atomicCAS(&g_debug_bounds[0], 0u, code) == 0u) {
+        g_debug_bounds[1] = static_cast<unsigned>(rb);
+        g_debug_bounds[2] = static_cast<unsigned>(cb);
+        g_debug_bounds[3] = static_cast<unsigned>(d.rows);
+        g_debug_bounds[4] = static_cast<unsigned>(d.cols);
+    }
+}
+#define CAME_DEBUG_SKIP_TILE(q) do { if ((q).skip) return; } while (0)
+#else
+#define CAME_DEBUG_SKIP_TILE(q) do { } while (0)
+#endif
 
 template <int VEC>
 __device__ __forceinline__ Geo make_geo(const TensorDev& d, int rb, int cb)
@@ -571,6 +595,21 @@ __device__ __forceinline__ Geo make_geo(const TensorDev& d, int rb, int cb)
     q.row0 = static_cast<long long>(rb) * d.tr;
     q.row1 = min(d.rows, q.row0 + d.tr);
     q.seg = cb * (TX >> 5) + (q.tx >> 5);
+    q.skip = false;
+#ifdef CAME_DEBUG_BOUNDS
+    unsigned bad = 0u;
+    if (rb < 0 || rb >= d.n_rb || q.row0 >= d.rows) bad = kDbgRowBlock;            // block-uniform
+    else if (cb < 0 || cb >= d.n_cb) bad = kDbgColBlock;                            // block-uniform
+    else if (q.row1 > d.rows || q.row1 - q.row0 > d.tr) bad = kDbgRowRange;         // block-uniform
+    else if (q.seg < 0 || q.seg >= d.n_seg) bad = kDbgSegment;                      // warp-uniform
+    else if (q.colok && q.col + VEC > d.cols) bad = kDbgVectorTail;                 // per thread
+    if (bad != 0u) {
+        debug_report(bad, d, rb, cb);
+        q.colok = false;                                     // this thread loads and stores nothing
+        if (bad != kDbgVectorTail) q.row1 = q.row0;          // whole warp: no rows, no row partials
+        q.skip = bad == kDbgRowBlock || bad == kDbgColBlock || bad == kDbgRowRange;
+    }
+#endif
     return q;
 }
 
@@ -677,6 +716,7 @@ __device__ __forceinline__ void p1_tile(const TensorDev& d, int rb, int cb, cons
     constexpr int VEC = Traits<KIND>::VEC;
     constexpr int U = UU > 0 ? UU : ((KIND == kF32x8) ? CAME_P12_U / 2 : CAME_P12_U);   // 32 raw registers either way
     const Geo q = make_geo<VEC>(d, rb, cb);
+    CAME_DEBUG_SKIP_TILE(q);
     const int lane = threadIdx.x & 31;
     const long long stride = static_cast<long long>(q.TY) * d.cols * grad_elem_bytes<KIND>();
     const char* gp = static_cast<const char*>(d.g) +
@@ -731,6 +771,7 @@ __device__ __forceinline__ void p2_tile(const TensorDev& d, int rb, int cb, cons
     constexpr int VEC = Traits<KIND>::VEC;
     constexpr int U = UU > 0 ? UU : ((KIND == kF32x8) ? CAME_P12_U / 2 : CAME_P12_U);   // 32 raw registers either way
     const Geo q = make_geo<VEC>(d, rb, cb);
+    CAME_DEBUG_SKIP_TILE(q);
     const long long stride = static_cast<long long>(q.TY) * d.cols * grad_elem_bytes<KIND>();
     const char* gp = static_cast<const char*>(d.g) +
                      ((q.row0 + q.ty) * d.cols + q.col) * grad_elem_bytes<KIND>();
@@ -786,6 +827,7 @@ __device__ __forceinline__ void p3_tile(const TensorDev& d, int rb, int cb, cons
     constexpr int VEC = Traits<KIND>::VEC;
     constexpr int U = UU > 0 ? UU : CAME_P34_U;
     const Geo q = make_geo<VEC>(d, rb, cb);
+    CAME_DEBUG_SKIP_TILE(q);
     const int lane = threadIdx.x & 31;
     const long long first = (q.row0 + q.ty) * d.cols + q.col;
     const long long gstride = static_cast<long long>(q.TY) * d.cols * grad_elem_bytes<KIND>();
@@ -868,6 +910,7 @@ __device__ __forceinline__ void p4_tile(const TensorDev& d, int rb, int cb, cons
     constexpr int VEC = Traits<KIND>::VEC;
     constexpr int U = UU > 0 ? UU : CAME_P34_U;
     const Geo q = make_geo<VEC>(d, rb, cb);
+    CAME_DEBUG_SKIP_TILE(q);
     if (!q.colok) return;
     const long long first = (q.row0 + q.ty) * d.cols + q.col;
     const long long stride = static_cast<long long>(q.TY) * d.cols;
@@ -925,6 +968,7 @@ __device__ __forceinline__ void p34_adafactor_tile(const TensorDev& d, int rb, i
     constexpr int VEC = Traits<KIND>::VEC;
     constexpr int U = UU > 0 ? UU : ((KIND == kF32x8) ? CAME_P34_U / 2 : CAME_P34_U);   // 24 registers per thread-row there
     const Geo q = make_geo<VEC>(d, rb, cb);
+    CAME_DEBUG_SKIP_TILE(q);
     if (!q.colok) return;
     const long long first = (q.row0 + q.ty) * d.cols + q.col;
     const long long gstride = static_cast<long long>(q.TY) * d.cols * grad_elem_bytes<KIND>();

@@ -193,6 +193,7 @@ __device__ __forceinline__ void stream_tile_p1(const TensorDev* __restrict__ T, 
     }
     const TensorDev d = T[cur.tensor];
     const Geo q = make_geo<VEC>(d, cur.rb, cur.cb);
+    CAME_DEBUG_SKIP_TILE(q);
     write_col_partials<VEC>(d, q, cur.rb, cacc, sm);
     finalize_factors(d, cur.rb, cur.cb, hc.beta2, hc.omb2, hc.eps1, hc.gscale2, d.r, d.c, d.scal + 0, sm);
     block_sync();          // the scratch is free again before the next tile's epilogue uses it

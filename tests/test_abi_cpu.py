@@ -227,3 +227,12 @@ def test_create_rejects_overlapping_buffers_without_cuda():
             binding.came_create([wide(grad=0x100000 + numel_bytes)])
         assert e.value.status == 7
     assert binding.came_status_string(12) == "CAME_ERR_OVERLAP"
+
+
+def test_debug_build_exports_the_same_symbols_and_ordinary_build_has_no_record():
+    L = binding.load_debug()
+    for n in _declared_functions():
+        assert hasattr(L, n), f"{n} missing from the bounds-checking build"
+    with pytest.raises(binding.CameError) as e:
+        binding.came_debug_bounds(0)                 # ordinary build: no record to read
+    assert e.value.status == 11
