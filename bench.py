@@ -280,7 +280,12 @@ def run_gpu(args):
         "roofline": roofline,
     }
     opt.close()
-    del opt, params, grads
+    del opt
+    if world == 1 and not args.no_configs and args.workload == "llama7b" and not ada:
+        # Algorithm 1 (Adafactor with momentum) on the same tensors: what the confidence term
+        # of Algorithm 2 costs on top of it (the paper: training time "increases only slightly")
+        line["algorithm1_mode"] = time_algorithm1(torch, binding, params, grads, hp, local_rank, ms_per_step)
+    del params, grads
     torch.cuda.empty_cache()
     if world == 1 and not args.no_configs and args.workload == "llama7b":
         # the other configurations, after the headline run has freed its memory: each is a
@@ -304,6 +309,28 @@ def _median(xs):
     xs = sorted(xs)
     n = len(xs)
     return xs[n // 2] if n % 2 else 0.5 * (xs[n // 2 - 1] + xs[n // 2])
+
+
+def time_algorithm1(torch, binding, params, grads, hp, device_index, came_ms, steps=10, warmup=3):
+    opt = binding.CameOptimizer(params, grads, device=device_index,
+                                create_flags=binding.CAME_CREATE_ADAFACTOR)
+    stream_bytes = opt.query(binding.CAME_Q_STREAM_BYTES)
+    for _ in range(warmup):
+        opt.step(**hp)
+    torch.cuda.synchronize()
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    marks[0].record()
+    for k in range(steps):
+        opt.step(**hp)
+        marks[k + 1].record()
+    torch.cuda.synchronize()
+    ms = _median([marks[k].elapsed_time(marks[k + 1]) for k in range(steps)])
+    numel = opt.query(binding.CAME_Q_NUMEL)
+    opt.close()
+    return {"ms_per_step_median": round(ms, 4), "params_per_s": numel / (ms * 1e-3),
+            "stream_bytes_per_step": stream_bytes,
+            "effective_GBps": round(stream_bytes / (ms * 1e-3) / 1e9, 1),
+            "came_over_algorithm1_time": round(came_ms / ms, 4), "steps": steps, "warmup": warmup}
 
 
 def time_config(torch, binding, name, device, peak, peak_kind, steps=20, warmup=5):
