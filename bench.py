@@ -161,6 +161,8 @@ def run_gpu(args):
     binding.load()                      # raises if the CUDA library cannot be had: no fallback
     binding.came_tune(binding.CAME_TUNE_SCHEDULE, {"default": 0, "phase": 1, "pipelined": 2}[args.schedule])
     binding.came_tune(binding.CAME_TUNE_SCHED_GROUP_BYTES, args.sched_group_bytes)
+    binding.came_tune(binding.CAME_TUNE_P1_STREAM, args.p1_stream)
+    binding.came_tune(binding.CAME_TUNE_P1_STREAM_RING, args.p1_stream_ring)
     binding.came_tune(binding.CAME_TUNE_PIPE_TILE_ELEMS, args.pipe_tile_elems)
     binding.came_tune(binding.CAME_TUNE_PIPE_GROUP_BYTES, args.pipe_group_bytes)
     w = synth.workload(args.workload)
@@ -597,6 +599,9 @@ def main():
                          "pipelined persistent grid")
     ap.add_argument("--sched-group-bytes", type=int, default=0,
                     help="phase grids launched group by group (CAME_TUNE_SCHED_GROUP_BYTES); 0 = off")
+    ap.add_argument("--p1-stream", type=int, default=0, choices=[0, 1, 2],
+                    help="CAME_TUNE_P1_STREAM: 2 = first phase as the persistent streaming grid")
+    ap.add_argument("--p1-stream-ring", type=int, default=0, help="CAME_TUNE_P1_STREAM_RING")
     ap.add_argument("--pipe-tile-elems", type=int, default=0, help="CAME_TUNE_PIPE_TILE_ELEMS")
     ap.add_argument("--pipe-group-bytes", type=int, default=0, help="CAME_TUNE_PIPE_GROUP_BYTES")
     ap.add_argument("--e2e-steps", type=int, default=2)
