@@ -317,8 +317,9 @@ came_status came_factor_update_static_plan(const void* grad, int32_t grad_dtype,
                                            double beta2, double eps1, int32_t device,
                                            int32_t* out_vec, int64_t* out_scratch_bytes);
 
-/* Process-wide tuning knobs, read by later came_create calls (plain globals: set them from
- * one thread, before the contexts they are meant for are created).  CAME_TUNE_TILE_ELEMS:
+/* Process-wide tuning knobs, read by later came_create calls (each knob is an atomic, so any
+ * thread may set one; a context takes the values in force while it is being created, so set
+ * them before the contexts they are meant for).  CAME_TUNE_TILE_ELEMS:
  * elements per matrix tile (0 restores the default, which scales with the size
  * of the parameter set).  They change scheduling only, never results beyond the
  * order of the partial sums. */

@@ -7,6 +7,7 @@
 #include "came_stream.cuh"
 
 #include <algorithm>
+#include <atomic>
 #include <cmath>
 #include <cstdio>
 #include <cstring>
@@ -26,25 +27,27 @@ const char* const kPhaseNames[kMaxPhases] = {
     "p1_reduce_g2", "p2_sum_u2", "p3_momentum_instability", "p4_apply", "p34_adafactor_apply"};
 
 thread_local std::string g_create_error;
-long long g_tile_elems_override = 0;   // came_tune(CAME_TUNE_TILE_ELEMS)
-bool g_use_pdl = true;                 // came_tune(CAME_TUNE_PDL)
-long long g_sched_group_bytes = 0;     // came_tune(CAME_TUNE_SCHED_GROUP_BYTES); 0 = one group
-long long g_host_group_bytes = 1ll << 30;   // came_tune(CAME_TUNE_HOST_GROUP_BYTES)
+// Tuning knobs (came_tune): process-wide, each one an atomic so that a knob set on one thread
+// is read whole on another; a context reads them once, while it is being created.
+std::atomic<long long> g_tile_elems_override{0};   // came_tune(CAME_TUNE_TILE_ELEMS)
+std::atomic<bool> g_use_pdl{true};                 // came_tune(CAME_TUNE_PDL)
+std::atomic<long long> g_sched_group_bytes{0};     // came_tune(CAME_TUNE_SCHED_GROUP_BYTES); 0 = one group
+std::atomic<long long> g_host_group_bytes{1ll << 30};   // came_tune(CAME_TUNE_HOST_GROUP_BYTES)
 
-int g_schedule = 0;                    // came_tune(CAME_TUNE_SCHEDULE): 0 auto, 1 phase grids, 2 pipelined
-long long g_pipe_tile_elems = 0;       // came_tune(CAME_TUNE_PIPE_TILE_ELEMS); 0 = default
-long long g_pipe_group_bytes = 0;      // came_tune(CAME_TUNE_PIPE_GROUP_BYTES); 0 = default
-long long g_pipe_wait_ns = 0;          // came_tune(CAME_TUNE_PIPE_WAIT_NS); 0 = default (2 s)
-long long g_pipe_order = 0;            // came_tune(CAME_TUNE_PIPE_ORDER)
+std::atomic<int> g_schedule{0};                    // came_tune(CAME_TUNE_SCHEDULE): 0 auto, 1 phase grids, 2 pipelined
+std::atomic<long long> g_pipe_tile_elems{0};       // came_tune(CAME_TUNE_PIPE_TILE_ELEMS); 0 = default
+std::atomic<long long> g_pipe_group_bytes{0};      // came_tune(CAME_TUNE_PIPE_GROUP_BYTES); 0 = default
+std::atomic<long long> g_pipe_wait_ns{0};          // came_tune(CAME_TUNE_PIPE_WAIT_NS); 0 = default (2 s)
+std::atomic<long long> g_pipe_order{0};            // came_tune(CAME_TUNE_PIPE_ORDER)
 constexpr long long kPipeTileElemsDefault = 32768;
 constexpr long long kPipeGroupBytesDefault = 48ll << 20;
 constexpr long long kPipeWaitNsDefault = 2000000000ll;
 
-int g_p1_stream = 0;                   // came_tune(CAME_TUNE_P1_STREAM): 0 default (off), 1 off, 2 on
-int g_p1_stream_ring = 0;              // came_tune(CAME_TUNE_P1_STREAM_RING): batches in the ring; 0 = default
+std::atomic<int> g_p1_stream{0};                   // came_tune(CAME_TUNE_P1_STREAM): 0 default (off), 1 off, 2 on
+std::atomic<int> g_p1_stream_ring{0};              // came_tune(CAME_TUNE_P1_STREAM_RING): batches in the ring; 0 = default
 constexpr int kP1StreamRingDefault = 2;
 
-bool g_f32_vec8 = true;                // came_tune(CAME_TUNE_F32_VEC8)
+std::atomic<bool> g_f32_vec8{true};                // came_tune(CAME_TUNE_F32_VEC8)
 inline bool g_f32_vec8_ok(bool bf) { return bf || g_f32_vec8; }
 
 struct Plan {
@@ -488,7 +491,8 @@ bool choose_pipelined(const came_tensor*, int)
 // sub-phases in between, which is what keeps the waits short.
 std::vector<came::Item> build_pipeline_items(came_ctx* ctx, const std::vector<Tile>& tiles)
 {
-    const long long group_bytes = g_pipe_group_bytes > 0 ? g_pipe_group_bytes : kPipeGroupBytesDefault;
+    const long long pipe_group = g_pipe_group_bytes.load();
+    const long long group_bytes = pipe_group > 0 ? pipe_group : kPipeGroupBytesDefault;
     auto resident = [](const came_tensor& x) {
         return x.rows * x.cols * (4ll + (x.grad_dtype == CAME_BF16 ? 2 : 4)); };
     const std::vector<Group> groups = make_groups(ctx, group_bytes, resident);
@@ -659,7 +663,7 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
     ctx->pipelined = choose_pipelined(t, n);
     long long target = g_tile_elems_override;
     if (target <= 0 && ctx->pipelined)
-        target = g_pipe_tile_elems > 0 ? g_pipe_tile_elems : kPipeTileElemsDefault;
+        target = g_pipe_tile_elems.load() > 0 ? g_pipe_tile_elems.load() : kPipeTileElemsDefault;
     if (target <= 0) {
         // aim for a few thousand tiles in all; between 4 Ki and 256 Ki elements per tile
         target = 4096;
@@ -764,8 +768,8 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
         CAME_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, came::k_step_pipelined,
                                                                came::kPipeThreads, 0), "occupancy query");
         ctx->pipe_grid = std::max(1, std::min(ctx->n_items, sms * std::max(per_sm, 1)));
-        ctx->pipe_wait_ns = static_cast<unsigned long long>(g_pipe_wait_ns > 0 ? g_pipe_wait_ns
-                                                                                : kPipeWaitNsDefault);
+        ctx->pipe_wait_ns = static_cast<unsigned long long>(g_pipe_wait_ns.load() > 0 ? g_pipe_wait_ns.load()
+                                                                                       : kPipeWaitNsDefault);
     }
     for (int k = 0; k < 2; ++k) {
         CAME_TRY(cudaMallocHost(&ctx->pinned_table[k], ctx->table_bytes), "cudaMallocHost(table)");
@@ -867,7 +871,7 @@ came_status came_create(came_ctx** out, const came_tensor* t, int32_t n, int32_t
             ctx->n_stream = static_cast<int>(n_st);
             ctx->n_others = static_cast<int>(others.size());
             ctx->p1_stream_ring = std::min(came::kStreamMaxBatches,
-                                           std::max(1, g_p1_stream_ring > 0 ? g_p1_stream_ring : kP1StreamRingDefault));
+                                           std::max(1, g_p1_stream_ring.load() > 0 ? g_p1_stream_ring.load() : kP1StreamRingDefault));
             const size_t ring_bytes = static_cast<size_t>(ctx->p1_stream_ring) * came::kStreamSlots * came::kThreads * 16;
             CAME_TRY(cudaFuncSetAttribute(came::k_p1_stream, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           static_cast<int>(ring_bytes)), "cudaFuncSetAttribute(ring)");
