@@ -411,13 +411,13 @@ def time_config(torch, binding, name, device, peak, peak_kind, steps=20, warmup=
 # (workload, kernel).  The figures belong to one build of the kernels: TRAFFIC_KERNEL_HASH is
 # kernel_source_hash() of the sources they were captured on, and traffic_bytes() answers None
 # (the JSON line then says "traffic": null) as soon as the sources differ.
-TRAFFIC_KERNEL_HASH = "eda8233e424708dc"
+TRAFFIC_KERNEL_HASH = "d64925ba8e73560c"
 TRAFFIC_BYTES = {
     # one-layer capture (profiles/ncu_phase_kernels_llama7b_layer.md) scaled by matrix elements
-    ("llama7b", "p4_apply"): 79.33e9,
-    ("llama7b", "p3_momentum_instability"): 66.75e9,
-    ("llama7b_layer", "p4_apply"): 2.3822e9,
-    ("llama7b_layer", "p3_momentum_instability"): 2.0046e9,
+    ("llama7b", "p4_apply"): 79.36e9,
+    ("llama7b", "p3_momentum_instability"): 66.78e9,
+    ("llama7b_layer", "p4_apply"): 2.3832e9,
+    ("llama7b_layer", "p3_momentum_instability"): 2.0055e9,
 }
 
 
