@@ -92,7 +92,8 @@ def test_shape_sweep_five_steps(env, shape):
 def test_bert_base_adafactor_mode(env):
     torch, binding, oracle = env
     w = synth.workload("bert_base")
-    _gate(run_paired(torch, binding, oracle, w, seed=2, steps=10, check_at=(1, 10), workers=WORKERS,
+    steps = _steps(w.steps, 10)             # all 100 steps with CAME_PARITY_FULL=1
+    _gate(run_paired(torch, binding, oracle, w, seed=2, steps=steps, check_at=(1, 10, steps), workers=WORKERS,
                      algorithm="adafactor"), "bert_base/adafactor")
 
 
